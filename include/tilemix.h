@@ -1,0 +1,155 @@
+/*
+ * tilemix.h -- C ABI of the TileMix hot path for NVIDIA B200 (sm_100a).
+ *
+ * TileMix (arxiv 2608.17336) is causal prefill attention in which every group of G adjacent
+ * key tiles of a query-tile row is routed, by one bit of a packed mask, to an FP16 or an
+ * INT8 QK^T score computation; both routes feed one shared online-softmax state, and the PV
+ * product stays FP16.  This library holds the three steps of that path:
+ *
+ *   tilemix_quantize_qk        blockwise symmetric INT8 quantiser for Q and K
+ *   tilemix_pack_routing_mask  routing map R -> packed words (+ coverage counters)
+ *   tilemix_attention_fwd      the fused mixed-precision attention kernel
+ *   tilemix_prefill_host       the three steps on HOST buffers (copies included)
+ *
+ * Conventions shared by every entry point
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer on the current CUDA
+ *     device; the caller owns every buffer; outputs are fully overwritten.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     No entry point allocates device memory or synchronises, except where stated.
+ *   - Return value: 0 = TILEMIX_OK; negative = a contract violation found on the host
+ *     BEFORE anything was launched; positive = the cudaError_t / CUresult of a failed
+ *     launch or tensor-map encode.  Nothing is printed, nothing throws.
+ *   - Indices are 0-based.  T_m = ceil(L/tile_m), T_n = ceil(L/tile_n),
+ *     T_mask = ceil(L/(G*tile_n)), W = ceil(T_mask/32).
+ */
+#ifndef TILEMIX_H_
+#define TILEMIX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TILEMIX_OK 0
+#define TILEMIX_ERR_NULL (-1)        /* a required pointer is NULL                          */
+#define TILEMIX_ERR_SHAPE (-2)       /* non-positive size, heads_q % heads_kv != 0, ...      */
+#define TILEMIX_ERR_UNSUPPORTED (-3) /* tile/head_dim combination or device not supported    */
+#define TILEMIX_ERR_ALIGN (-4)       /* base pointer or stride not 16-byte aligned           */
+#define TILEMIX_ERR_WORKSPACE (-5)   /* workspace / arena smaller than required              */
+#define TILEMIX_ERR_DEVICE_TIMEOUT (-6) /* reported by tilemix_read_status only              */
+
+/* flags of tilemix_problem_t */
+#define TILEMIX_FORCE_FP16 1u /* ignore the mask: every tile takes the FP16 route; the INT8
+                                 operands, scales and mask may then be NULL               */
+/* pack_flags of tilemix_pack_routing_mask */
+#define TILEMIX_PIN_DIAGONAL_FP16 1u
+
+/* Shape of one attention call, in the paper's notation (Sec. 3.1, Sec. 4.1): B, H_q, H_k,
+ * L = L_q = L_k, d, BLOCK_M x BLOCK_N score tiles, g key tiles per routing bit.
+ * Strides are in elements, for (batch, head, token); the head_dim axis is contiguous.  A
+ * stride triple of all zeros means dense [B, H, L, d].  INT8 operands, scales, mask words
+ * and the routing map are always dense. */
+typedef struct tilemix_problem {
+    int32_t batch, heads_q, heads_kv, seqlen, head_dim;
+    int32_t tile_m, tile_n;           /* routing / quantisation tile; supported: 64x64 with
+                                         head_dim 64, 128x128 with head_dim 128             */
+    int32_t group;                    /* G >= 1                                              */
+    int32_t quant_blk_q, quant_blk_k; /* rows per scale; 0 = tile_m / tile_n                 */
+    int32_t mask_batch;               /* 1 = one mask shared by the batch, or == batch       */
+    uint32_t flags;
+    float softmax_scale;              /* <= 0 means 1/sqrt(head_dim)                         */
+    int32_t reserved;
+    int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];
+} tilemix_problem_t;
+
+/* Debug request for tilemix_attention_fwd: the raw score accumulators of the listed tiles. */
+typedef struct tilemix_debug {
+    const int32_t* tiles; /* [n_tiles, 4] = (b, h_q, m, n), legal tiles (n <= m)            */
+    int32_t n_tiles;
+    int32_t* raw;         /* [n_tiles, tile_m, tile_n]: INT8-routed tile: the INT32
+                             accumulator Q8_m K8_n^T exactly as the tensor core produced it
+                             (before scaling and masking; rows/cols beyond L are 0);
+                             FP16-routed tile: the bit pattern of the FP32 accumulator      */
+    uint8_t* kind;        /* [n_tiles]: 1 = INT32 written, 0 = FP32 bits written             */
+} tilemix_debug_t;
+
+/* Blockwise symmetric INT8 quantisation of Q and K (App. C, "Blockwise INT8 Quantization"
+ * and "Quantization Granularity"): for every block r of quant_blk rows of one head,
+ * delta = max|x| / 127 and xhat = round(x / delta) in {-127..127}, computed in FP32 with
+ * IEEE division and round-half-to-even; a zero block gives delta = 0, xhat = 0; a tail block
+ * takes its maximum over the rows that exist.
+ *   q_f16 [B,Hq,L,d], k_f16 [B,Hk,L,d]  FP16, strided per the problem
+ *   q_i8, k_i8                          INT8, dense, same shapes
+ *   q_scale [B,Hq,ceil(L/blk_q)], k_scale [B,Hk,ceil(L/blk_k)]  FP32
+ * Either operand may be skipped by passing all three of its pointers as NULL. */
+int tilemix_quantize_qk(const tilemix_problem_t* p, const void* q_f16, const void* k_f16,
+                        int8_t* q_i8, int8_t* k_i8, float* q_scale, float* k_scale,
+                        void* stream);
+
+/* Packed routing words (Sec. 4.2, "Bitmask packing"): for every (nb, h_k, m) the word row
+ * b = sum_g R[g] * 2^g, stored as W little-endian uint32 words (group g -> word g>>5,
+ * bit g&31; for T_mask <= 64 this is the paper's one 64-bit word).  1 = INT8, 0 = FP16.
+ * Bits of groups with no legal (query, key) pair, of pad positions >= T_mask and -- with
+ * TILEMIX_PIN_DIAGONAL_FP16 -- of groups holding a key tile that straddles the diagonal are
+ * written as 0.
+ *   route      uint8 [nb, Hk, T_m, T_mask], non-zero = INT8
+ *   mask_words uint32 [nb, Hk, T_m, W]
+ *   counts     nullable uint64 [nb, Hk, 2] = {legal groups, INT8-routed legal groups}
+ *              (App. B, "Coverage Accounting") */
+int tilemix_pack_routing_mask(const tilemix_problem_t* p, const uint8_t* route,
+                              uint32_t pack_flags, uint32_t* mask_words, uint64_t* counts,
+                              void* stream);
+
+/* The fused kernel (Sec. 4.1 loops, Sec. 4.3 "Tile-group dispatch", App. C): for every query
+ * tile m it streams key tiles n <= m; bit floor(n/G) of row (h_k, m) selects
+ *   S = Q_m K_n^T / sqrt(d)                                   (FP16 route, bit 0) or
+ *   S = delta_Q[m] delta_K[n] (Q8_m K8_n^T) / sqrt(d)         (INT8 route, bit 1),
+ * both update one FP32 online-softmax state (Sec. 3.1), P is rounded to FP16 for the PV
+ * product, and O = O~/z is written as FP16.  h_k = h_q / (H_q/H_k).
+ *   lse        nullable float [B,Hq,L]: max + ln(sum) of the scaled scores of each row
+ *   workspace  >= tilemix_workspace_size(p) bytes, 16-byte aligned; its first 16 bytes are a
+ *              status record (see tilemix_read_status) which this call clears on the stream
+ *   dbg        nullable; see tilemix_debug_t
+ * Requires quant_blk_q == tile_m and quant_blk_k == tile_n, 16-byte aligned bases and
+ * strides, and a device of compute capability 10.0. */
+int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const void* k_f16,
+                          const void* v_f16, const int8_t* q_i8, const int8_t* k_i8,
+                          const float* q_scale, const float* k_scale,
+                          const uint32_t* mask_words, void* out_f16, float* lse,
+                          void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg,
+                          void* stream);
+
+/* Whole path on HOST buffers: copies Q, K, V and the routing map to the device arena,
+ * quantises, packs, runs the fused kernel and copies O back; everything is enqueued on
+ * `stream` in order (use pinned host memory for the copies to be asynchronous).
+ *   q_host,k_host,v_host  host FP16, dense [B,H,L,d];  route_host host uint8 [nb,Hk,T_m,T_mask]
+ *   out_host              host FP16, dense [B,Hq,L,d]
+ *   arena                 device scratch of >= tilemix_arena_size(p) bytes, 256-byte aligned */
+int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const void* k_host,
+                         const void* v_host, const uint8_t* route_host, uint32_t pack_flags,
+                         void* out_host, void* arena, size_t arena_bytes, void* stream);
+
+/* W = ceil(ceil(L / (G*tile_n)) / 32); <= 0 on invalid arguments. */
+int tilemix_mask_words_per_row(int seqlen, int tile_n, int group);
+/* Bytes of `workspace` needed by tilemix_attention_fwd (0 on an invalid problem). */
+size_t tilemix_workspace_size(const tilemix_problem_t* p);
+/* Bytes of the quantize-once scratch of App. D's accounting: INT8 Q and K, their FP32
+ * scales and the packed words (0 on an invalid problem). */
+size_t tilemix_scratch_bytes(const tilemix_problem_t* p);
+/* Bytes of `arena` needed by tilemix_prefill_host (0 on an invalid problem). */
+size_t tilemix_arena_size(const tilemix_problem_t* p);
+/* Synchronises `stream`, then copies the 4-word status record of the last
+ * tilemix_attention_fwd on that workspace to host `out`: {code, role, tile index, barrier}.
+ * Returns out[0]: TILEMIX_OK or TILEMIX_ERR_DEVICE_TIMEOUT (a bounded wait inside the kernel
+ * ran out; the outputs of that call are then undefined). */
+int tilemix_read_status(const void* workspace, int32_t out[4], void* stream);
+const char* tilemix_status_string(int code);
+/* Number of kernels this library has launched since it was loaded (all entry points). */
+uint64_t tilemix_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TILEMIX_H_ */

@@ -82,6 +82,7 @@ def _load():
         build()
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_init()
     return _lib
 
 

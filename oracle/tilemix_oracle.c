@@ -45,7 +45,7 @@ typedef struct {
 } oracle_problem_t;
 
 /* IEEE binary16 -> binary32, exact (every half is representable as a float). */
-static float half_bits_to_float(uint16_t h) {
+static float decode_half(uint16_t h) {
     uint32_t sign = (uint32_t)(h >> 15) & 1u;
     uint32_t expo = (uint32_t)(h >> 10) & 0x1fu;
     uint32_t frac = (uint32_t)h & 0x3ffu;
@@ -59,6 +59,18 @@ static float half_bits_to_float(uint16_t h) {
     }
     return sign ? -v : v;
 }
+
+/* The 65536 decoded values, tabulated once (decode_half is the definition). */
+static float g_half_table[65536];
+static int g_half_table_ready = 0;
+
+void oracle_init(void) {
+    if (g_half_table_ready) return;
+    for (uint32_t h = 0; h < 65536u; ++h) g_half_table[h] = decode_half((uint16_t)h);
+    g_half_table_ready = 1;
+}
+
+static float half_bits_to_float(uint16_t h) { return g_half_table[h]; }
 
 static int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 

@@ -1,0 +1,252 @@
+// C ABI of libtilemix: argument validation on the host, then the kernel launchers.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace tilemix {
+
+std::atomic<uint64_t> g_launch_count{0};
+
+namespace {
+
+bool all_zero(const int64_t s[3]) { return s[0] == 0 && s[1] == 0 && s[2] == 0; }
+
+void dense_strides(int H, int L, int d, int64_t out[3]) {
+    out[0] = static_cast<int64_t>(H) * L * d;
+    out[1] = static_cast<int64_t>(L) * d;
+    out[2] = d;
+}
+
+int set_strides(const int64_t in[3], int H, int L, int d, int64_t out[3]) {
+    if (all_zero(in)) {
+        dense_strides(H, L, d, out);
+        return TILEMIX_OK;
+    }
+    for (int i = 0; i < 3; ++i) {
+        if (in[i] < 0) return TILEMIX_ERR_SHAPE;
+        out[i] = in[i];
+    }
+    if (out[2] < d) return TILEMIX_ERR_SHAPE;
+    // 16-byte granularity of FP16 rows (vector loads and TMA global strides)
+    for (int i = 0; i < 3; ++i)
+        if ((out[i] * 2) % 16 != 0) return TILEMIX_ERR_ALIGN;
+    return TILEMIX_OK;
+}
+
+int check_device() {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    return major == 10 ? TILEMIX_OK : TILEMIX_ERR_UNSUPPORTED;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+int resolve(const tilemix_problem_t* p, Geometry* g) {
+    if (p == nullptr) return TILEMIX_ERR_NULL;
+    if (p->batch <= 0 || p->heads_q <= 0 || p->heads_kv <= 0 || p->seqlen <= 0 || p->head_dim <= 0 ||
+        p->tile_m <= 0 || p->tile_n <= 0 || p->group <= 0)
+        return TILEMIX_ERR_SHAPE;
+    if (p->heads_q % p->heads_kv != 0) return TILEMIX_ERR_SHAPE;
+    if (p->head_dim % 8 != 0) return TILEMIX_ERR_SHAPE;
+    if (p->mask_batch != 1 && p->mask_batch != p->batch) return TILEMIX_ERR_SHAPE;
+    if (p->quant_blk_q < 0 || p->quant_blk_k < 0) return TILEMIX_ERR_SHAPE;
+    g->B = p->batch; g->Hq = p->heads_q; g->Hk = p->heads_kv; g->L = p->seqlen; g->d = p->head_dim;
+    g->tile_m = p->tile_m; g->tile_n = p->tile_n; g->G = p->group;
+    g->blk_q = p->quant_blk_q ? p->quant_blk_q : p->tile_m;
+    g->blk_k = p->quant_blk_k ? p->quant_blk_k : p->tile_n;
+    g->nb = p->mask_batch;
+    g->T_m = static_cast<int>(ceil_div(g->L, g->tile_m));
+    g->T_n = static_cast<int>(ceil_div(g->L, g->tile_n));
+    g->T_mask = static_cast<int>(ceil_div(g->L, static_cast<int64_t>(g->G) * g->tile_n));
+    g->W = static_cast<int>(ceil_div(g->T_mask, 32));
+    g->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(g->d));
+    g->flags = p->flags;
+    int rc;
+    if ((rc = set_strides(p->q_stride, g->Hq, g->L, g->d, g->qs))) return rc;
+    if ((rc = set_strides(p->k_stride, g->Hk, g->L, g->d, g->ks))) return rc;
+    if ((rc = set_strides(p->v_stride, g->Hk, g->L, g->d, g->vs))) return rc;
+    if ((rc = set_strides(p->o_stride, g->Hq, g->L, g->d, g->os))) return rc;
+    return TILEMIX_OK;
+}
+
+}  // namespace tilemix
+
+using namespace tilemix;
+
+extern "C" {
+
+int tilemix_quantize_qk(const tilemix_problem_t* p, const void* q_f16, const void* k_f16, int8_t* q_i8,
+                        int8_t* k_i8, float* q_scale, float* k_scale, void* stream) {
+    Geometry g;
+    int rc = resolve(p, &g);
+    if (rc) return rc;
+    const bool do_q = q_f16 || q_i8 || q_scale, do_k = k_f16 || k_i8 || k_scale;
+    if (!do_q && !do_k) return TILEMIX_ERR_NULL;
+    if (do_q && !(q_f16 && q_i8 && q_scale)) return TILEMIX_ERR_NULL;
+    if (do_k && !(k_f16 && k_i8 && k_scale)) return TILEMIX_ERR_NULL;
+    if ((do_q && (!aligned16(q_f16) || !aligned16(q_i8))) || (do_k && (!aligned16(k_f16) || !aligned16(k_i8))))
+        return TILEMIX_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (do_q && (rc = launch_quantize(q_f16, g.qs, g.B, g.Hq, g.L, g.d, g.blk_q, q_i8, q_scale, s))) return rc;
+    if (do_k && (rc = launch_quantize(k_f16, g.ks, g.B, g.Hk, g.L, g.d, g.blk_k, k_i8, k_scale, s))) return rc;
+    return TILEMIX_OK;
+}
+
+int tilemix_pack_routing_mask(const tilemix_problem_t* p, const uint8_t* route, uint32_t pack_flags,
+                              uint32_t* mask_words, uint64_t* counts, void* stream) {
+    Geometry g;
+    int rc = resolve(p, &g);
+    if (rc) return rc;
+    if (route == nullptr || mask_words == nullptr) return TILEMIX_ERR_NULL;
+    return launch_pack(g, route, pack_flags, mask_words, reinterpret_cast<unsigned long long*>(counts),
+                       static_cast<cudaStream_t>(stream));
+}
+
+int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const void* k_f16, const void* v_f16,
+                          const int8_t* q_i8, const int8_t* k_i8, const float* q_scale, const float* k_scale,
+                          const uint32_t* mask_words, void* out_f16, float* lse, void* workspace,
+                          size_t workspace_bytes, const tilemix_debug_t* dbg, void* stream) {
+    Geometry g;
+    int rc = resolve(p, &g);
+    if (rc) return rc;
+    if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
+    const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
+    if (!force16 && !(q_i8 && k_i8 && q_scale && k_scale && mask_words)) return TILEMIX_ERR_NULL;
+    if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
+    if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
+    const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
+                          (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
+    if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.W > 64) return TILEMIX_ERR_UNSUPPORTED;
+    if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
+        !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
+        (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
+        return TILEMIX_ERR_ALIGN;
+    if (workspace_bytes < tilemix_workspace_size(p)) return TILEMIX_ERR_WORKSPACE;
+    if ((rc = check_device())) return rc;
+    return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
+                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+}
+
+int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {
+    if (seqlen <= 0 || tile_n <= 0 || group <= 0) return TILEMIX_ERR_SHAPE;
+    const int64_t t_mask = ceil_div(seqlen, static_cast<int64_t>(tile_n) * group);
+    return static_cast<int>(ceil_div(t_mask, 32));
+}
+
+size_t tilemix_workspace_size(const tilemix_problem_t* p) {
+    Geometry g;
+    if (resolve(p, &g)) return 0;
+    return 256;   // status record (16 bytes used)
+}
+
+size_t tilemix_scratch_bytes(const tilemix_problem_t* p) {
+    Geometry g;
+    if (resolve(p, &g)) return 0;
+    const size_t int8 = static_cast<size_t>(g.B) * g.L * g.d * (static_cast<size_t>(g.Hq) + g.Hk);
+    const size_t scales = 4u * static_cast<size_t>(g.B) *
+                          (static_cast<size_t>(g.Hq) * ceil_div(g.L, g.blk_q) + static_cast<size_t>(g.Hk) * ceil_div(g.L, g.blk_k));
+    const size_t words = 4u * static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.W;
+    return int8 + scales + words;
+}
+
+namespace {
+// Layout of the arena used by tilemix_prefill_host (every region 256-byte aligned).
+struct Arena {
+    size_t q, k, v, o, q8, k8, qs, ks, route, words, work, total;
+};
+Arena arena_layout(const Geometry& g) {
+    Arena a;
+    size_t off = 0;
+    auto put = [&](size_t bytes) { const size_t at = off; off = align_up(off + bytes, 256); return at; };
+    const size_t nq = static_cast<size_t>(g.B) * g.Hq * g.L * g.d, nk = static_cast<size_t>(g.B) * g.Hk * g.L * g.d;
+    a.q = put(nq * 2); a.k = put(nk * 2); a.v = put(nk * 2); a.o = put(nq * 2);
+    a.q8 = put(nq); a.k8 = put(nk);
+    a.qs = put(4u * static_cast<size_t>(g.B) * g.Hq * ceil_div(g.L, g.blk_q));
+    a.ks = put(4u * static_cast<size_t>(g.B) * g.Hk * ceil_div(g.L, g.blk_k));
+    a.route = put(static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.T_mask);
+    a.words = put(4u * static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.W);
+    a.work = put(256);
+    a.total = off;
+    return a;
+}
+}  // namespace
+
+size_t tilemix_arena_size(const tilemix_problem_t* p) {
+    Geometry g;
+    if (resolve(p, &g)) return 0;
+    return arena_layout(g).total;
+}
+
+int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const void* k_host, const void* v_host,
+                         const uint8_t* route_host, uint32_t pack_flags, void* out_host, void* arena,
+                         size_t arena_bytes, void* stream) {
+    Geometry g;
+    int rc = resolve(p, &g);
+    if (rc) return rc;
+    if (!q_host || !k_host || !v_host || !route_host || !out_host || !arena) return TILEMIX_ERR_NULL;
+    if (!all_zero(p->q_stride) || !all_zero(p->k_stride) || !all_zero(p->v_stride) || !all_zero(p->o_stride))
+        return TILEMIX_ERR_UNSUPPORTED;   // host buffers are dense
+    if (reinterpret_cast<uintptr_t>(arena) % 256 != 0) return TILEMIX_ERR_ALIGN;
+    const Arena a = arena_layout(g);
+    if (arena_bytes < a.total) return TILEMIX_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(arena);
+    const size_t nq = static_cast<size_t>(g.B) * g.Hq * g.L * g.d, nk = static_cast<size_t>(g.B) * g.Hk * g.L * g.d;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(base + a.q, q_host, nq * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+    if ((e = cudaMemcpyAsync(base + a.k, k_host, nk * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+    if ((e = cudaMemcpyAsync(base + a.v, v_host, nk * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+    if ((e = cudaMemcpyAsync(base + a.route, route_host, static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.T_mask,
+                             cudaMemcpyHostToDevice, s)) != cudaSuccess)
+        return e;
+    tilemix_problem_t dense = *p;
+    if ((rc = tilemix_quantize_qk(&dense, base + a.q, base + a.k, reinterpret_cast<int8_t*>(base + a.q8),
+                                  reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
+                                  reinterpret_cast<float*>(base + a.ks), stream)))
+        return rc;
+    if ((rc = tilemix_pack_routing_mask(&dense, base + a.route, pack_flags, reinterpret_cast<uint32_t*>(base + a.words),
+                                        nullptr, stream)))
+        return rc;
+    if ((rc = tilemix_attention_fwd(&dense, base + a.q, base + a.k, base + a.v, reinterpret_cast<int8_t*>(base + a.q8),
+                                    reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
+                                    reinterpret_cast<float*>(base + a.ks), reinterpret_cast<uint32_t*>(base + a.words),
+                                    base + a.o, nullptr, base + a.work, 256, nullptr, stream)))
+        return rc;
+    if ((e = cudaMemcpyAsync(out_host, base + a.o, nq * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return e;
+    return TILEMIX_OK;
+}
+
+int tilemix_read_status(const void* workspace, int32_t out[4], void* stream) {
+    if (!workspace || !out) return TILEMIX_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(out, workspace, 16, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    return out[0];
+}
+
+const char* tilemix_status_string(int code) {
+    switch (code) {
+        case TILEMIX_OK: return "ok";
+        case TILEMIX_ERR_NULL: return "a required pointer is NULL";
+        case TILEMIX_ERR_SHAPE: return "invalid shape";
+        case TILEMIX_ERR_UNSUPPORTED: return "unsupported tile/head_dim combination or device";
+        case TILEMIX_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+        case TILEMIX_ERR_WORKSPACE: return "workspace too small";
+        case TILEMIX_ERR_DEVICE_TIMEOUT: return "a bounded wait inside the kernel ran out";
+        default: return code > 0 ? cudaGetErrorString(static_cast<cudaError_t>(code)) : "unknown";
+    }
+}
+
+uint64_t tilemix_launch_count(void) { return g_launch_count.load(); }
+
+}  // extern "C"

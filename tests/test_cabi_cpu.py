@@ -1,0 +1,112 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every symbol the public header
+declares, rejects bad arguments on the host before any launch, and its size helpers agree
+with the closed forms of the paper's accounting."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_17336_b200 import binding as b
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_17336_b200 import build
+    build.build()
+    return b.lib()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    declared = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        text = open(os.path.join(ROOT, "include", fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        declared |= set(re.findall(r"\b(tilemix_[a-z0-9_]+)\s*\(", text))
+    assert declared == set(b.EXPORTS), declared ^ set(b.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_problem_struct_matches_header_layout():
+    assert ctypes.sizeof(b.ProblemStruct) == 14 * 4 + 12 * 8
+    assert b.ProblemStruct.q_stride.offset == 56 and b.ProblemStruct.o_stride.offset == 56 + 72
+
+
+def _args(n):
+    return [ctypes.c_void_p(0x1000)] * n
+
+
+def test_host_side_validation_without_gpu(lib):
+    good = b.problem(1, 2, 2, 1024, 128, 128, 128)
+    null = None
+    # NULL problem / pointers
+    assert lib.tilemix_quantize_qk(None, *_args(6), null) == b.ERR_NULL
+    assert lib.tilemix_quantize_qk(ctypes.byref(good), null, null, null, null, null, null, null) == b.ERR_NULL
+    assert lib.tilemix_quantize_qk(ctypes.byref(good), ctypes.c_void_p(0x1000), null, null, null, null, null, null) == b.ERR_NULL
+    assert lib.tilemix_pack_routing_mask(ctypes.byref(good), null, 0, ctypes.c_void_p(0x1000), null, null) == b.ERR_NULL
+    # shapes
+    for field, val in (("batch", 0), ("seqlen", -1), ("group", 0), ("heads_kv", 3), ("head_dim", 12), ("mask_batch", 2)):
+        bad = b.problem(1, 2, 2, 1024, 128, 128, 128)
+        setattr(bad, field, val)
+        assert lib.tilemix_quantize_qk(ctypes.byref(bad), *_args(6), null) == b.ERR_SHAPE, field
+        assert lib.tilemix_workspace_size(ctypes.byref(bad)) == 0
+    # alignment of bases and strides
+    assert lib.tilemix_quantize_qk(ctypes.byref(good), ctypes.c_void_p(0x1008), *_args(5), null) == b.ERR_ALIGN
+    odd = b.problem(1, 2, 2, 1024, 128, 128, 128)
+    odd.q_stride[0], odd.q_stride[1], odd.q_stride[2] = 2 * 1024 * 132, 1024 * 132, 132
+    assert lib.tilemix_quantize_qk(ctypes.byref(odd), *_args(6), null) == b.ERR_ALIGN
+    # attention: unsupported tile / head_dim / quant block, missing INT8 operands, small workspace
+    att = lambda p, ws=256, q8=0x1000: lib.tilemix_attention_fwd(
+        ctypes.byref(p), *_args(3), ctypes.c_void_p(q8) if q8 else None, *_args(5), None, ctypes.c_void_p(0x1000), ws, None, None)
+    assert att(b.problem(1, 2, 2, 1024, 128, 64, 64)) == b.ERR_UNSUPPORTED
+    assert att(b.problem(1, 2, 2, 1024, 96, 128, 128)) == b.ERR_UNSUPPORTED
+    assert att(b.problem(1, 2, 2, 1024, 128, 128, 128, quant_blk_k=64)) == b.ERR_UNSUPPORTED
+    assert att(good, ws=8) == b.ERR_WORKSPACE
+    assert att(good, q8=0) == b.ERR_NULL
+    assert att(good, q8=0x1001) == b.ERR_ALIGN
+    dbg = b.DebugStruct(None, 3, None, None)
+    assert lib.tilemix_attention_fwd(ctypes.byref(good), *_args(9), None, ctypes.c_void_p(0x1000), 256,
+                                     ctypes.byref(dbg), None) == b.ERR_NULL
+    assert lib.tilemix_launch_count() == 0
+
+
+def test_status_strings(lib):
+    for code in (0, -1, -2, -3, -4, -5, -6):
+        assert lib.tilemix_status_string(code)
+    assert b"wait" in lib.tilemix_status_string(b.ERR_DEVICE_TIMEOUT)
+
+
+def test_mask_words_per_row(lib):
+    assert b.tilemix_mask_words_per_row(1024, 64, 1) == 1
+    assert b.tilemix_mask_words_per_row(8192, 128, 1) == 2
+    assert b.tilemix_mask_words_per_row(32768, 128, 4) == 2
+    assert b.tilemix_mask_words_per_row(4096, 128, 2) == 1
+    assert b.tilemix_mask_words_per_row(131072, 128, 8) == 4
+    assert b.tilemix_mask_words_per_row(0, 128, 8) < 0
+    for L, t, g in ((1000, 128, 3), (77, 64, 1), (5000, 64, 2)):
+        assert b.tilemix_mask_words_per_row(L, t, g) == oracle.Problem(1, 1, 1, L, 64, t, t, g).W
+
+
+def test_scratch_bytes_matches_paper_accounting(lib):
+    """App. D accounting shape (H_q=32, H_k=8, L=8192, d=128, BLK_Q=128, BLK_K=64): the
+    quantize-once scratch is everything beyond the FP16 Q/K/V; with this library's FP32 scales
+    and two uint32 words per row it is the closed form with 4-byte scales and 8-byte rows."""
+    p = b.problem(1, 32, 8, 8192, 128, 128, 128, 1, quant_blk_q=128, quant_blk_k=64)
+    total, fp16 = oracle.resident_bytes_quantize_once(32, 8, 8192, 128, 128, 64, 128, scale_bytes=4, word_bytes=8)
+    assert b.tilemix_scratch_bytes(p) == total - fp16
+    # and with the paper's FP16 scales the same sum is the printed 136.01 MiB
+    total16, _ = oracle.resident_bytes_quantize_once(32, 8, 8192, 128, 128, 64, 128)
+    assert round(total16 / 2 ** 20, 2) == 136.01
+    assert b.tilemix_arena_size(p) >= total
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(b, "_lib", None)
+    monkeypatch.setattr(b, "LIB_PATH", "/nonexistent/libtilemix.so")
+    with pytest.raises(RuntimeError, match="no CPU or library fallback"):
+        b.lib()

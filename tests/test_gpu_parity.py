@@ -1,0 +1,269 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs:
+bit-exact for INT8 operands, scales, packed words, counters and INT32 score accumulators;
+FP16 outputs within 2e-3 * max(1, |O|)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_17336_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2608_17336_b200 import binding
+    return binding
+
+
+def _small(name, **kw):
+    base = dict(name=name, batch=1, heads=2, seqlen=640, head_dim=128, tile=128, group=1, seed=11,
+                routing="bernoulli", int8_fraction=0.5)
+    base.update(kw)
+    return synth.Workload(**base)
+
+
+# ------------------------------------------------------------------------------ quantiser
+
+@pytest.mark.parametrize("B,Hh,L,d,blk", [(1, 2, 640, 128, 128), (2, 3, 1000, 128, 128), (1, 1, 1024, 64, 64),
+                                         (1, 2, 100, 64, 64), (1, 1, 777, 128, 64), (1, 2, 300, 32, 16)])
+def test_quantize_bit_exact(B, Hh, L, d, blk):
+    b = _binding()
+    gen = torch.Generator().manual_seed(L + d)
+    q = (torch.randn((B, Hh, L, d), generator=gen) * 3).half()
+    k = torch.randn((B, Hh, L, d), generator=gen).half()
+    k[0, 0, : min(L, 2 * blk)] = 0          # zero blocks
+    p = b.problem(B, Hh, Hh, L, d, blk, blk)
+    q8, k8, qs, ks = b.tilemix_quantize_qk(p, q.cuda(), k.cuda())
+    for x, x8, xs in ((q, q8, qs), (k, k8, ks)):
+        r8, rs = oracle.quantize(H.np_bits(x), blk)
+        assert (x8.cpu().numpy() == r8).all()
+        assert (xs.cpu().numpy().view(np.uint32) == rs.view(np.uint32)).all()
+
+
+def test_quantize_strided_input():
+    b = _binding()
+    B, Hh, L, d = 2, 3, 384, 128
+    gen = torch.Generator().manual_seed(5)
+    packed = torch.randn((B, L, 3, Hh, d), generator=gen).half().cuda()    # a fused QKV projection output
+    q = packed[:, :, 0].permute(0, 2, 1, 3)                                # [B, H, L, d] view, d contiguous
+    k = packed[:, :, 1].permute(0, 2, 1, 3)
+    p = b.problem(B, Hh, Hh, L, d, 128, 128)
+    q8, k8, qs, ks = b.tilemix_quantize_qk(p, q, k)
+    r8, rs = oracle.quantize(H.np_bits(q.contiguous().cpu()), 128)
+    assert (q8.cpu().numpy() == r8).all() and (qs.cpu().numpy() == rs).all()
+    r8, rs = oracle.quantize(H.np_bits(k.contiguous().cpu()), 128)
+    assert (k8.cpu().numpy() == r8).all() and (ks.cpu().numpy() == rs).all()
+
+
+# ------------------------------------------------------------------------------ packer
+
+@pytest.mark.parametrize("L,tile,G,nb,pin", [(1024, 64, 1, 1, False), (8192, 128, 1, 1, False), (32768, 128, 4, 1, True),
+                                             (4096, 128, 2, 2, False), (131072, 128, 8, 1, False), (1000, 128, 3, 1, True),
+                                             (100, 64, 1, 1, True)])
+def test_pack_bit_exact(L, tile, G, nb, pin):
+    b = _binding()
+    Hk = 3
+    p = b.problem(nb, Hk, Hk, L, tile, tile, tile, G, mask_batch=nb)
+    rng = np.random.default_rng(L + G)
+    route = (rng.random((nb, Hk, p.T_m, p.T_mask)) < 0.7).astype(np.uint8) * rng.integers(1, 255, 1, dtype=np.uint8)
+    words, counts = b.tilemix_pack_routing_mask(p, torch.from_numpy(route).cuda(), pin)
+    po = oracle.Problem(nb, Hk, Hk, L, tile, tile, tile, G, mask_batch=nb)
+    rw, rc = oracle.pack(po, route, pin)
+    assert (words.cpu().numpy().view(np.uint32) == rw).all()
+    assert (counts.cpu().numpy().astype(np.uint64) == rc).all()
+
+
+# ------------------------------------------------------------------------------ attention
+
+def _full_check(w, debug=True, atol=H.ATOL):
+    q, k, v = synth.make_qkv(w)
+    route = synth.make_route(w)
+    heads = list(range(w.heads))
+    rows = H.all_rows(w)
+    ref = H.run_oracle(w, q, k, v, route, heads, rows)
+    tiles = None
+    if debug:
+        tiles = [(b, h, m, n) for b in range(w.batch) for h in heads for m in range(w.T_m) for n in range(m + 1)]
+    res = H.run_gpu(w, q, k, v, route, debug_tiles=tiles)
+    # bit-exact parts
+    assert (res["q8"].cpu().numpy() == ref["q8"]).all() and (res["k8"].cpu().numpy() == ref["k8"]).all()
+    assert (res["qs"].cpu().numpy() == ref["qs"]).all() and (res["ks"].cpu().numpy() == ref["ks"]).all()
+    assert (res["words"].cpu().numpy().view(np.uint32) == ref["words"]).all()
+    assert (res["counts"].cpu().numpy().astype(np.uint64) == ref["counts"]).all()
+    if debug:
+        raw = res["raw"].cpu().numpy()
+        kind = res["kind"].cpu().numpy()
+        po = ref["p"]
+        n_int8 = 0
+        for e, (b, h, m, n) in enumerate(tiles):
+            g = n // w.group
+            nbi = 0 if w.mask_batch == 1 else b
+            bit = (int(ref["words"][nbi, h, m, g >> 5]) >> (g & 31)) & 1
+            assert kind[e] == bit, (b, h, m, n, kind[e], bit)
+            if bit:
+                n_int8 += 1
+                exp = oracle.int32_tile(po, ref["q8"], ref["k8"], b, h, m, n)
+                assert (raw[e] == exp).all(), f"INT32 accumulator tile {(b, h, m, n)} differs"
+            else:
+                exp = oracle.fp_tile(po, ref["qb"], ref["kb"], b, h, m, n)
+                got = raw[e].view(np.float32).astype(np.float64)
+                assert np.abs(got - exp).max() <= 1e-3 * max(1.0, np.abs(exp).max()), (b, h, m, n)
+        assert w.routing in ("zero",) or n_int8 > 0
+    err = H.check_rows(res["out"], ref["out"], rows, atol)
+    lse = res["lse"].cpu().numpy().astype(np.float64).reshape(-1)
+    assert np.abs(lse - ref["lse"]).max() < 2e-3
+    return err
+
+
+def test_attention_cfg1_tiny_all_rows_all_int32_tiles():
+    """Config 1 in full: every row against the oracle, all 136 raw accumulator tiles bit-exact."""
+    _full_check(synth.WORKLOADS["cfg1_tiny"])
+
+
+@pytest.mark.parametrize("routing,frac", [("zero", 0.0), ("one", 1.0), ("bernoulli", 0.5)])
+def test_attention_small_d128(routing, frac):
+    _full_check(_small("s128", routing=routing, int8_fraction=frac))
+
+
+def test_attention_odd_tile_count_grouped_mask():
+    _full_check(_small("odd", seqlen=896, group=2, heads=1, seed=12))          # 7 tiles: last pair has no B
+
+
+def test_attention_ragged_tail():
+    _full_check(_small("ragged", seqlen=1000, group=3, seed=13, pin_diagonal=True))
+    _full_check(_small("ragged64", seqlen=333, head_dim=64, tile=64, group=2, seed=14))
+
+
+def test_attention_single_partial_tile():
+    _full_check(_small("one_tile", seqlen=100, heads=1, seed=15))
+    _full_check(_small("one_row", seqlen=1, heads=1, seed=16))
+
+
+def test_attention_batched_mask_per_batch_and_outliers():
+    _full_check(_small("batched", batch=2, heads=2, seqlen=512, mask_batch=2, values="outlier_channels", seed=17))
+
+
+def test_attention_force_fp16_without_int8_operands():
+    b = _binding()
+    w = _small("force16", routing="zero", seqlen=512)
+    q, k, v = synth.make_qkv(w)
+    p = H.gpu_problem(w, flags=b.FORCE_FP16)
+    res = b.tilemix_attention_fwd(p, q.cuda(), k.cuda(), v.cuda())
+    assert b.tilemix_read_status(res["workspace"])[0] == 0
+    rows = H.all_rows(w)
+    ref = H.run_oracle(w, q, k, v, synth.make_route(w), range(w.heads), rows)
+    H.check_rows(res["out"], ref["out"], rows)
+
+
+def test_attention_gqa_heads_share_kv_and_mask():
+    """H_q = 4, H_k = 2: h_k = floor(h_q / 2) indexes K, V, K8, scales and the routing words."""
+    b = _binding()
+    B, Hq, Hk, L, d, tile = 1, 4, 2, 512, 128, 128
+    gen = torch.Generator().manual_seed(21)
+    q = torch.randn((B, Hq, L, d), generator=gen).half()
+    k = torch.randn((B, Hk, L, d), generator=gen).half()
+    v = torch.randn((B, Hk, L, d), generator=gen).half()
+    p = b.problem(B, Hq, Hk, L, d, tile, tile, 1)
+    po = oracle.Problem(B, Hq, Hk, L, d, tile, tile, 1)
+    route = (np.random.default_rng(3).random((1, Hk, po.T_m, po.T_mask)) < 0.5).astype(np.uint8)
+    q8, k8, qs, ks = b.tilemix_quantize_qk(p, q.cuda(), k.cuda())
+    words, _ = b.tilemix_pack_routing_mask(p, torch.from_numpy(route).cuda())
+    res = b.tilemix_attention_fwd(p, q.cuda(), k.cuda(), v.cuda(), q8, k8, qs, ks, words)
+    assert b.tilemix_read_status(res["workspace"])[0] == 0
+    oq8, oqs = oracle.quantize(H.np_bits(q), tile)
+    ok8, oks = oracle.quantize(H.np_bits(k), tile)
+    ow, _ = oracle.pack(po, route)
+    ref, _, _ = oracle.attention_full(po, H.np_bits(q), H.np_bits(k), H.np_bits(v), oq8, ok8, oqs, oks, ow)
+    err = np.abs(res["out"].float().cpu().numpy() - ref)
+    assert (err <= H.ATOL * np.maximum(1, np.abs(ref))).all(), err.max()
+
+
+def test_attention_strided_qkv_views():
+    b = _binding()
+    B, Hh, L, d = 1, 2, 512, 128
+    gen = torch.Generator().manual_seed(23)
+    packed = torch.randn((B, L, 3, Hh, d), generator=gen).half()
+    q, k, v = (packed[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    w = _small("strided", seqlen=L, heads=Hh)
+    route = synth.make_route(w)
+    p = H.gpu_problem(w)
+    pd = packed.cuda()
+    qd, kd, vd = (pd[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    q8, k8, qs, ks = b.tilemix_quantize_qk(p, qd, kd)
+    words, _ = b.tilemix_pack_routing_mask(p, torch.from_numpy(route).cuda())
+    res = b.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words)
+    assert b.tilemix_read_status(res["workspace"])[0] == 0
+    rows = H.all_rows(w)
+    ref = H.run_oracle(w, q.contiguous(), k.contiguous(), v.contiguous(), route, range(Hh), rows)
+    H.check_rows(res["out"], ref["out"], rows)
+
+
+def test_lossless_inputs_every_mask_equals_fp16():
+    """Q, K on the grid {-127..127}/64 with +-127/64 in every block quantise exactly, so every
+    routing map must reproduce the all-FP16 result (up to summation order)."""
+    b = _binding()
+    w = _small("lossless", seqlen=768, heads=1, group=2)
+    gen = torch.Generator().manual_seed(31)
+    shape = (1, 1, w.seqlen, 128)
+    q = torch.randint(-127, 128, shape, generator=gen).float()
+    k = torch.randint(-127, 128, shape, generator=gen).float()
+    q[..., ::128, 0] = 127; k[..., ::128, 0] = -127
+    q, k = (q / 64).half(), (k / 64).half()
+    v = torch.randn(shape, generator=gen).half()
+    outs = []
+    for routing in ("zero", "one", "bernoulli"):
+        res = H.run_gpu(w.scaled(routing=routing), q, k, v, synth.make_route(w.scaled(routing=routing)))
+        assert (res["qs"] == 1 / 64).all() and (res["ks"] == 1 / 64).all()
+        outs.append(res["out"].float())
+    assert (outs[0] - outs[1]).abs().max() < 1e-3 and (outs[0] - outs[2]).abs().max() < 1e-3
+
+
+def test_two_runs_are_bit_identical():
+    w = _small("repeat", seqlen=1024, heads=2)
+    q, k, v = synth.make_qkv(w)
+    route = synth.make_route(w)
+    a = H.run_gpu(w, q, k, v, route)["out"]
+    c = H.run_gpu(w, q, k, v, route)["out"]
+    assert torch.equal(a, c)
+
+
+# ------------------------------------------------------------------------------ full-size configs
+
+FULL = [
+    ("cfg2_llama8k", dict(routing="zero"), 2, 2, 16),
+    ("cfg2_llama8k", dict(), 2, 2, 16),
+    ("cfg2_llama8k", dict(routing="one"), 2, 2, 16),
+    ("cfg3_long32k", dict(), 2, 1, 8),
+    ("cfg4_batched4k", dict(), 3, 2, 16),
+    ("cfg5_verylong128k", dict(), 1, 0, 6),
+]
+
+
+@pytest.mark.parametrize("name,override,n_heads,n_tiles,n_rows", FULL)
+def test_full_size_config_sampled_rows(name, override, n_heads, n_tiles, n_rows):
+    """The five configurations at full size, in the launch configuration the bench times; the oracle
+    evaluates sampled rows of a few heads (first and last query tile, random tiles, random rows)."""
+    w = synth.WORKLOADS[name].scaled(**override)
+    q, k, v = synth.make_qkv(w)
+    route = synth.make_route(w)
+    heads = sorted({0, w.heads - 1, w.heads // 2})[:n_heads]
+    rows = synth.sample_rows(w, n_random_tiles=n_tiles, n_random_rows=n_rows, heads=heads)
+    if w.seqlen > 40000:      # keep the oracle to seconds: only a few rows of the last (longest) tile
+        keep = (rows[:, 2] < w.seqlen - w.tile) | (rows[:, 2] % 16 == 15)
+        rows = rows[keep]
+    if w.batch > 1:
+        rows = rows[(rows[:, 0] == 0) | (rows[:, 0] == w.batch - 1)]
+    res = H.run_gpu(w, q, k, v, route, want_lse=False)
+    ref = H.run_oracle(w, q, k, v, route, heads, [tuple(r) for r in rows])
+    sub = torch.as_tensor(heads)
+    assert (res["q8"][:, sub].cpu().numpy() == ref["q8"]).all() and (res["k8"][:, sub].cpu().numpy() == ref["k8"]).all()
+    assert (res["qs"][:, sub].cpu().numpy() == ref["qs"]).all() and (res["ks"][:, sub].cpu().numpy() == ref["ks"]).all()
+    assert (res["words"][:, sub].cpu().numpy().view(np.uint32) == ref["words"]).all()
+    H.check_rows(res["out"], ref["out"], rows)
+    # properties that hold at any size: finite outputs, |O| bounded by max |V| of the head
+    out = res["out"]
+    assert torch.isfinite(out).all()
+    vmax = v.abs().amax(dim=(2, 3)).cuda()
+    assert (out.abs().amax(dim=(2, 3)) <= vmax * (1 + 1e-2)).all()
