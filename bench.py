@@ -153,6 +153,7 @@ def main():
     ap.add_argument("--int8-fraction", type=float, default=None, help="override the workload's INT8 coverage")
     ap.add_argument("--ref-pairs", type=float, default=6e7, help="oracle sample size (query-key pairs per step)")
     ap.add_argument("--cpu-pairs", type=float, default=4e8, help="cpu_baseline sample size (pairs)")
+    ap.add_argument("--heads", type=int, default=None, help="override the head count (smaller profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -162,6 +163,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     w = synth.WORKLOADS[args.workload]
+    if args.heads is not None:
+        w = w.scaled(heads=args.heads)
     if args.int8_fraction is not None:
         routing = "zero" if args.int8_fraction <= 0 else "one" if args.int8_fraction >= 1 else w.routing
         w = w.scaled(int8_fraction=args.int8_fraction, routing=routing)

@@ -137,8 +137,9 @@ def test_attention_ragged_tail():
 
 
 def test_attention_single_partial_tile():
-    _full_check(_small("one_tile", seqlen=100, heads=1, seed=15))
-    _full_check(_small("one_row", seqlen=1, heads=1, seed=16))
+    _full_check(_small("one_tile", seqlen=100, heads=1, seed=15, routing="one"))
+    _full_check(_small("one_tile16", seqlen=100, heads=1, seed=15, routing="zero"))
+    _full_check(_small("one_row", seqlen=1, heads=1, seed=16, routing="one"))
 
 
 def test_attention_batched_mask_per_batch_and_outliers():
