@@ -37,6 +37,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, f) for f in SOURCES]
+    cmd += os.environ.get("TILEMIX_NVCC_FLAGS", "").split()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

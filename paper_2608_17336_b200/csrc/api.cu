@@ -124,7 +124,7 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
                           (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
     if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
     if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.W > 64) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
     if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
         !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
         (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
@@ -144,7 +144,7 @@ int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {
 size_t tilemix_workspace_size(const tilemix_problem_t* p) {
     Geometry g;
     if (resolve(p, &g)) return 0;
-    return 256;   // status record (16 bytes used)
+    return 1024;   // status record (16 bytes) + optional phase timers
 }
 
 size_t tilemix_scratch_bytes(const tilemix_problem_t* p) {
@@ -173,7 +173,7 @@ Arena arena_layout(const Geometry& g) {
     a.ks = put(4u * static_cast<size_t>(g.B) * g.Hk * ceil_div(g.L, g.blk_k));
     a.route = put(static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.T_mask);
     a.words = put(4u * static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.W);
-    a.work = put(256);
+    a.work = put(1024);
     a.total = off;
     return a;
 }
@@ -218,7 +218,7 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
     if ((rc = tilemix_attention_fwd(&dense, base + a.q, base + a.k, base + a.v, reinterpret_cast<int8_t*>(base + a.q8),
                                     reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
                                     reinterpret_cast<float*>(base + a.ks), reinterpret_cast<uint32_t*>(base + a.words),
-                                    base + a.o, nullptr, base + a.work, 256, nullptr, stream)))
+                                    base + a.o, nullptr, base + a.work, 1024, nullptr, stream)))
         return rc;
     if ((e = cudaMemcpyAsync(out_host, base + a.o, nq * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return e;
     return TILEMIX_OK;

@@ -32,7 +32,8 @@ constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kThreads = 320;
 constexpr int kRing = 8;
-constexpr int kMaxWords = 64;             // packed words per row kept in shared memory
+constexpr int kWorkspaceClearBytes = 1024;  // status record + optional phase timers
+constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -65,7 +66,7 @@ struct Cfg {
     static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1;
     static constexpr int kOffMisc = kOffBars + kNumBars * 8;       // tmem base, abort flag
     static constexpr int kOffWords = kOffMisc + 16;
-    static constexpr int kSmemBytes = kOffWords + 2 * kMaxWords * 4;
+    static constexpr int kSmemBytes = kOffWords + kMaxTiles / 2;   // 4-bit schedule entries
     static constexpr int kSmemAlloc = kSmemBytes + 1024;           // slack to align the base
     static_assert(kK8Bytes <= kChunk, "INT8 key tile must fit one ring chunk");
     static_assert(kTmemCols == 256 || kTmemCols == 512, "TMEM allocation must be a power of two");
@@ -95,6 +96,17 @@ struct Ctx {
     int* status;
 };
 
+// Optional phase timers (compile with -DTILEMIX_PHASE_TIMERS): cycles spent in each bounded wait,
+// summed over all CTAs into 64-bit counters that follow the status record in the workspace
+// (index = role * 8 + barrier kind; 32.. = whole-CTA and softmax-loop totals).  Only the first
+// thread of each role contributes.
+#ifdef TILEMIX_PHASE_TIMERS
+#define TM_TIMER_ADD(idx, cycles) atomicAdd(reinterpret_cast<unsigned long long*>(cx.status) + 8 + (idx), \
+                                            static_cast<unsigned long long>(cycles))
+#else
+#define TM_TIMER_ADD(idx, cycles) ((void)0)
+#endif
+
 __device__ __forceinline__ void record_timeout(const Ctx& cx, int role, int tile, int which) {
     *cx.abort_flag = 1;
     if (atomicCAS(&cx.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
@@ -108,6 +120,9 @@ __device__ __forceinline__ void record_timeout(const Ctx& cx, int role, int tile
 __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, int role,
                                          int tile, int which) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
+#ifdef TILEMIX_PHASE_TIMERS
+    const long long c0 = clock64();
+#endif
     const uint64_t t0 = ptx::globaltimer_ns();
     uint32_t it = 0;
     while (!ptx::mbar_try_wait(bar, parity)) {
@@ -119,6 +134,9 @@ __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t p
             }
         }
     }
+#ifdef TILEMIX_PHASE_TIMERS
+    if ((threadIdx.x & 127) == 0 || role >= kRoleProducer) TM_TIMER_ADD(role * 8 + which, clock64() - c0);
+#endif
     return true;
 }
 
@@ -143,9 +161,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-__device__ __forceinline__ uint32_t route_bit(const uint32_t* row_words, int n, int G) {
-    const int g = n / G;
-    return (row_words[g >> 5] >> (g & 31)) & 1u;
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
 template <int D, int T>
@@ -165,6 +190,9 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     __syncthreads();
     if (s_skip != 0) return;
 
+#ifdef TILEMIX_PHASE_TIMERS
+    const long long cta_c0 = clock64();
+#endif
     // ---- work item -------------------------------------------------------------------
     const int n_pairs = (prm.T_m + 1) >> 1;
     const int bh = blockIdx.x / n_pairs;
@@ -185,7 +213,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     auto bar_o = [&](int t) { return bar0 + 8u * (6 + 2 * kRing + t); };
     const uint32_t bar_drain = bar0 + 8u * (8 + 2 * kRing);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);   // [0] tmem base, [1] abort
-    uint32_t* words_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
+    uint32_t* sched_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
     Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status};
 
     if (threadIdx.x == 0) {
@@ -204,16 +232,28 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         misc[1] = 0;
         ptx::fence_mbar_init();
     }
-    // routing words of rows A and B (zeros = FP16 everywhere)
-    for (int i = threadIdx.x; i < 2 * kMaxWords; i += kThreads) {
-        const int t = i / kMaxWords, w = i - t * kMaxWords;
-        const int m = t ? mB : mA;
-        uint32_t v = 0u;
-        if (prm.words != nullptr && w < prm.W && m < prm.T_m) {
-            const int nbi = (prm.nb == 1) ? 0 : b;
-            v = prm.words[((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.T_m + m) * prm.W + w];
+    // Schedule table, one 4-bit entry per key tile j (Sec. 4.2 lookup done once per CTA):
+    //   bit0 / bit1: tile A / tile B takes the INT8 route at key tile j  (R = (b >> floor(j/G)) & 1)
+    //   bit2 / bit3: the FP16 / the INT8 copy of K_j has to be staged
+    for (int i = threadIdx.x; i * 8 < nkv; i += kThreads) {
+        uint32_t packed = 0u;
+        for (int jj = 0; jj < 8; ++jj) {
+            const int j = i * 8 + jj;
+            if (j >= nkv) break;
+            uint32_t e = 0u;
+            if (prm.words != nullptr) {
+                const int g = j / prm.G;
+                const int nbi = (prm.nb == 1) ? 0 : b;
+                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.T_m + mA) * prm.W;
+                e |= (rowA[g >> 5] >> (g & 31)) & 1u;
+                if (hasB) e |= ((rowA[prm.W + (g >> 5)] >> (g & 31)) & 1u) << 1;
+            }
+            const bool useA = j <= mA;
+            if ((useA && !(e & 1u)) || (hasB && !(e & 2u))) e |= 4u;
+            if ((useA && (e & 1u)) || (hasB && (e & 2u))) e |= 8u;
+            packed |= e << (4 * jj);
         }
-        words_s[i] = v;
+        sched_s[i] = packed;
     }
     if (warp == kMmaWarp) {
         ptx::tmem_alloc(ptx::smem_u32(&misc[0]), C::kTmemCols);
@@ -223,16 +263,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc[0];
-    const uint32_t* wordsA = words_s;
-    const uint32_t* wordsB = words_s + kMaxWords;
-
-    // which K operands key tile j must bring: bit0 = FP16 copy, bit1 = INT8 copy
-    auto k_needs = [&](int j) -> uint32_t {
-        uint32_t need = 0u;
-        if (j <= mA) need |= route_bit(wordsA, j, prm.G) ? 2u : 1u;
-        if (hasB) need |= route_bit(wordsB, j, prm.G) ? 2u : 1u;
-        return need;
-    };
+    auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
     if (warp == kProducerWarp) {
         // ================================================================ TMA producer
@@ -254,32 +285,31 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (prm.has_int8)
                     ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, m * T, hq, b);
             }
+            // One ring item = the chunks of one operand tile.  Its data arrives on the "full" barrier
+            // of its first chunk; every chunk is handed back on its own "empty" barrier (items of
+            // different sizes reuse the chunks in different groupings).
             Ring ring;
             ring.phases = 0xffu;   // first wait on every "empty" barrier passes immediately
             uint32_t issued = 0u, full_phase = 0u, last_parity = 0u;   // per-slot bits
             bool ok = true;
-            auto fill = [&](uint32_t s, const CUtensorMap* tm, uint32_t bytes, int c0, int row) {
-                if (!ok) return;
-                if (!wait_bar(cx, bar_empty(s), ring.phase(s), kRoleProducer, row / T, kBarRingEmpty)) {
-                    ok = false;
-                    return;
+            auto fill = [&](uint32_t s, int n_chunks, const CUtensorMap* tm, uint32_t bytes, int row) {
+                for (int c = 0; c < n_chunks && ok; ++c) {
+                    if (!wait_bar(cx, bar_empty(s + c), ring.phase(s + c), kRoleProducer, row / T, kBarRingEmpty)) ok = false;
+                    ring.flip(s + c);
                 }
-                ring.flip(s);
+                if (!ok) return;
                 ptx::mbar_arrive_expect_tx(bar_full(s), bytes);
-                ptx::tma_load_4d(sbase + C::kOffRing + s * C::kChunk, tm, bar_full(s), c0, row, hk, b);
+                for (int c = 0; c < n_chunks; ++c)
+                    ptx::tma_load_4d(sbase + C::kOffRing + (s + c) * C::kChunk, tm, bar_full(s), c * 64, row, hk, b);
                 last_parity = (last_parity & ~(1u << s)) | (full_phase & (1u << s));
                 full_phase ^= 1u << s;
                 issued |= 1u << s;
             };
             for (int j = 0; j < nkv && ok; ++j) {
-                const uint32_t need = k_needs(j);
-                if (need & 1u) {
-                    const uint32_t s = ring.take(C::kHalves);
-                    for (int c = 0; c < C::kHalves; ++c) fill(s + c, &tm_k16, C::kChunk, c * 64, j * T);
-                }
-                if (need & 2u) fill(ring.take(1), &tm_k8, C::kK8Bytes, 0, j * T);
-                const uint32_t s = ring.take(C::kHalves);
-                for (int c = 0; c < C::kHalves; ++c) fill(s + c, &tm_v16, C::kChunk, c * 64, j * T);
+                const uint32_t e = sched(j);
+                if (e & 4u) fill(ring.take(C::kHalves), C::kHalves, &tm_k16, C::kHalves * C::kChunk, j * T);
+                if (e & 8u) fill(ring.take(1), 1, &tm_k8, C::kK8Bytes, j * T);
+                fill(ring.take(C::kHalves), C::kHalves, &tm_v16, C::kHalves * C::kChunk, j * T);
             }
             if (!ok || *cx.abort_flag) {
                 // let copies that are still in flight land before the CTA's memory is released
@@ -303,27 +333,36 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (!wait_bar(cx, bar_full(s), ring.phase(s), kRoleMma, j, kBarRingFull)) ok = false;
                 ring.flip(s);
             };
+            // Descriptor words that do not change: the high words, and the low words of the
+            // resident Q operands.  One K step advances a K-major operand by 32 bytes inside its
+            // swizzle atom (+2 in the low word) and the MN-major V operand by 16 keys = 2048 bytes.
+            constexpr uint32_t kHi16 = ptx::desc_hi(1024, 2);
+            constexpr uint32_t kHi8 = ptx::desc_hi(C::kI8Sbo, C::kI8Layout);
+            const uint32_t ring_lo = ptx::desc_lo(sbase + C::kOffRing, 16);
+            const uint32_t ring_lo_v = ptx::desc_lo(sbase + C::kOffRing, C::kChunk);
+            constexpr uint32_t kChunkLo = C::kChunk >> 4;
             // S_t = Q_t K_j^T on the route of tile t
             auto issue_qk = [&](int t, uint32_t int8_route, uint32_t s16, uint32_t s8) {
                 const uint32_t d_tmem = tmem_base + t * C::kSCols;
                 if (int8_route) {
-                    const uint32_t a0 = sbase + C::kOffQ8 + t * C::kQ8Tile;
-                    const uint32_t b0 = sbase + C::kOffRing + s8 * C::kChunk;
+                    const uint32_t a_lo = ptx::desc_lo(sbase + C::kOffQ8 + t * C::kQ8Tile, 16);
+                    const uint32_t b_lo = ring_lo + s8 * kChunkLo;
+                    ptx::mma_i8_ss<false>(d_tmem, a_lo, kHi8, b_lo, kHi8, kIdescQK8);
 #pragma unroll
-                    for (int k = 0; k < D / 32; ++k)
-                        ptx::mma_i8_ss(d_tmem, ptx::smem_desc(a0 + k * 32, 16, C::kI8Sbo, C::kI8Layout),
-                                       ptx::smem_desc(b0 + k * 32, 16, C::kI8Sbo, C::kI8Layout), kIdescQK8,
-                                       k > 0);
+                    for (int k = 1; k < D / 32; ++k)
+                        ptx::mma_i8_ss<true>(d_tmem, a_lo + 2 * k, kHi8, b_lo + 2 * k, kHi8, kIdescQK8);
                 } else {
 #pragma unroll
                     for (int c = 0; c < C::kHalves; ++c) {
-                        const uint32_t a0 = sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab;
-                        const uint32_t b0 = sbase + C::kOffRing + (s16 + c) * C::kChunk;
+                        const uint32_t a_lo = ptx::desc_lo(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, 16);
+                        const uint32_t b_lo = ring_lo + (s16 + c) * kChunkLo;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            ptx::mma_f16_ss(d_tmem, ptx::smem_desc(a0 + k * 32, 16, 1024, 2),
-                                            ptx::smem_desc(b0 + k * 32, 16, 1024, 2), kIdescQK16,
-                                            (c | k) > 0);
+                        for (int k = 0; k < 4; ++k) {
+                            if (c == 0 && k == 0)
+                                ptx::mma_f16_ss<false>(d_tmem, a_lo, kHi16, b_lo, kHi16, kIdescQK16);
+                            else
+                                ptx::mma_f16_ss<true>(d_tmem, a_lo + 2 * k, kHi16, b_lo + 2 * k, kHi16, kIdescQK16);
+                        }
                     }
                 }
             };
@@ -331,63 +370,74 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             auto issue_pv = [&](int t, uint32_t sv, uint32_t accumulate) {
                 const uint32_t d_tmem = tmem_base + 2 * C::kSCols + t * C::kOCols;
                 const uint32_t a_tmem = tmem_base + t * C::kSCols;
-                const uint32_t b0 = sbase + C::kOffRing + sv * C::kChunk;
+                const uint32_t b_lo = ring_lo_v + sv * kChunkLo;
+                ptx::mma_f16_ts(d_tmem, a_tmem, b_lo, kHi16, kIdescPV, accumulate);
 #pragma unroll
-                for (int k = 0; k < T / 16; ++k)
-                    ptx::mma_f16_ts(d_tmem, a_tmem + k * 8, ptx::smem_desc(b0 + k * 2048, C::kChunk, 1024, 2),
-                                    kIdescPV, accumulate | (k > 0));
+                for (int k = 1; k < T / 16; ++k)
+                    ptx::mma_f16_ts(d_tmem, a_tmem + k * 8, b_lo + k * 128, kHi16, kIdescPV, 1u);
             };
 
             for (int t = 0; t < (hasB ? 2 : 1) && ok; ++t)
                 if (!wait_bar(cx, bar_q(t), 0, kRoleMma, t, kBarQ)) ok = false;
 
             // slots of the K operands of the tile whose QK^T is issued next
-            uint32_t need = k_needs(0), k16 = 0, k8 = 0;
-            if (need & 1u) { k16 = ring.take(C::kHalves); for (int c = 0; c < C::kHalves; ++c) acquire(k16 + c, 0); }
-            if (need & 2u) { k8 = ring.take(1); acquire(k8, 0); }
+            uint32_t e_next = sched(0), k16 = 0, k8 = 0;
+            if (e_next & 4u) { k16 = ring.take(C::kHalves); acquire(k16, 0); }
+            if (e_next & 8u) { k8 = ring.take(1); acquire(k8, 0); }
             if (ok) {
                 ptx::tc_fence_after_sync();
-                issue_qk(0, route_bit(wordsA, 0, prm.G), k16, k8);
+                issue_qk(0, e_next & 1u, k16, k8);
                 ptx::mma_commit(bar_s(0));
                 if (hasB) {
-                    issue_qk(1, route_bit(wordsB, 0, prm.G), k16, k8);
+                    issue_qk(1, e_next & 2u, k16, k8);
                     ptx::mma_commit(bar_s(1));
                 }
-                if (need & 1u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
-                if (need & 2u) ptx::mma_commit(bar_empty(k8));
+                if (e_next & 4u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
+                if (e_next & 8u) ptx::mma_commit(bar_empty(k8));
             }
             for (int j = 0; j < nkv && ok; ++j) {
                 const uint32_t sv = ring.take(C::kHalves);
-                const bool more = j + 1 < nkv;
-                need = more ? k_needs(j + 1) : 0u;
-                if (need & 1u) k16 = ring.take(C::kHalves);
-                if (need & 2u) k8 = ring.take(1);
-                bool v_ready = false, k_ready = false;
-                for (int t = 0; t < 2 && ok; ++t) {
+                e_next = (j + 1 < nkv) ? sched(j + 1) : 0u;
+                if (e_next & 4u) k16 = ring.take(C::kHalves);
+                if (e_next & 8u) k8 = ring.take(1);
+                // operands of this iteration: wait for them now, off the P -> PV critical path
+                acquire(sv, j);
+                if (e_next & 4u) acquire(k16, j + 1);
+                if (e_next & 8u) acquire(k8, j + 1);
+                if (!ok) break;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
                     const int m_t = t ? mB : mA;
                     if ((t == 1 && !hasB) || j > m_t) continue;
+#ifdef TILEMIX_PHASE_TIMERS
+                    const long long mw0 = clock64();
+#endif
                     if (!wait_bar(cx, bar_p(t), j & 1, kRoleMma, j, kBarP)) { ok = false; break; }
-                    if (!v_ready) { for (int c = 0; c < C::kHalves; ++c) acquire(sv + c, j); v_ready = true; }
-                    if (!ok) break;
+#ifdef TILEMIX_PHASE_TIMERS
+                    const long long mw1 = clock64();
+                    TM_TIMER_ADD(45, mw1 - mw0);
+#endif
                     ptx::tc_fence_after_sync();
                     issue_pv(t, sv, j > 0);
                     if (j == m_t) ptx::mma_commit(bar_o(t));
+#ifdef TILEMIX_PHASE_TIMERS
+                    const long long mw3 = clock64();
+#endif
                     if (j + 1 <= m_t) {
-                        if (!k_ready) {
-                            if (need & 1u) for (int c = 0; c < C::kHalves; ++c) acquire(k16 + c, j + 1);
-                            if (need & 2u) acquire(k8, j + 1);
-                            k_ready = true;
-                            if (!ok) break;
-                            ptx::tc_fence_after_sync();
-                        }
-                        issue_qk(t, route_bit(t ? wordsB : wordsA, j + 1, prm.G), k16, k8);
+                        issue_qk(t, e_next & (1u << t), k16, k8);
                         ptx::mma_commit(bar_s(t));
                     }
+#ifdef TILEMIX_PHASE_TIMERS
+                    const long long mw5 = clock64();
+                    TM_TIMER_ADD(46, mw5 - mw1);
+                    TM_TIMER_ADD(47, 1);
+                    TM_TIMER_ADD(49, mw3 - mw1); TM_TIMER_ADD(51, mw5 - mw3);
+#endif
                 }
                 if (!ok) break;
                 for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(sv + c));
-                if (need & 1u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
-                if (need & 2u) ptx::mma_commit(bar_empty(k8));
+                if (e_next & 4u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
+                if (e_next & 8u) ptx::mma_commit(bar_empty(k8));
             }
             // every MMA issued by this thread has retired before TMEM / shared memory go away
             ptx::mma_commit(bar_drain);
@@ -403,7 +453,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const uint32_t t_s = lane_base + t * C::kSCols;
             const uint32_t t_o = lane_base + 2 * C::kSCols + t * C::kOCols;
-            const uint32_t* words_t = t ? wordsB : wordsA;
             const int64_t i_glob = static_cast<int64_t>(m_t) * T + row;
             const bool row_valid = row < T && i_glob < prm.L;
             const float dq = prm.has_int8 ? prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t] : 0.f;
@@ -412,23 +461,38 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
 
+#ifdef TILEMIX_PHASE_TIMERS
+            const long long loop_c0 = clock64();
+#endif
             for (int j = 0; j <= m_t; ++j) {
-                const uint32_t int8_route = route_bit(words_t, j, prm.G);
+                const uint32_t int8_route = (sched(j) >> t) & 1u;
                 float a = prm.scale_log2;
                 if (int8_route) {
                     a *= dq * dk_row[j];
                     if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                 }
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long sw0 = clock64();
+#endif
                 ok = wait_bar(cx, bar_s(t), j & 1, role, j, kBarS);
+#ifdef TILEMIX_PHASE_TIMERS
+                if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(39, clock64() - sw0);
+#endif
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long st0 = clock64();
+#endif
 
                 uint32_t s[T];
 #pragma unroll
                 for (int c = 0; c < T / 32; ++c)
                     ptx::tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
                 ptx::tmem_wait_ld();
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long st1 = clock64();
+#endif
 
                 if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
                     int idx = -1;
@@ -448,35 +512,109 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     }
                 }
 
-                // common score domain: FP32 raw accumulators (App. C), then causal legality
-                float mx = -INFINITY;
+                // Row maximum of the raw accumulators.  The scale a is >= 0, so max(a*raw) =
+                // a*max(raw); for INT8 tiles the maximum is taken on the integers.
                 const bool diag = (j == m_t);
+                float mx;
+                if (diag) {
+                    // Diagonal tile (one per row of tiles): generic path.  Convert to FP32 and
+                    // apply causal legality (App. B: enforced kernel-side, independent of R).
+                    mx = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < T; ++c) {
-                    float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
-                    if (diag && c > row) v = -INFINITY;
-                    s[c] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
+                    for (int c = 0; c < T; ++c) {
+                        float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
+                        if (c > row) v = -INFINITY;
+                        s[c] = __float_as_uint(v);
+                        mx = fmaxf(mx, v);
+                    }
+                } else if (int8_route) {
+                    int mi[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) mi[u] = static_cast<int>(s[u]);
+#pragma unroll
+                    for (int c = 4; c < T - 4; c += 8) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            mi[u] = __vimax3_s32(mi[u], static_cast<int>(s[c + 2 * u]), static_cast<int>(s[c + 2 * u + 1]));
+                    }
+                    // (T - 4) % 8 == 4: the last four columns
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) mi[u] = max(mi[u], static_cast<int>(s[T - 4 + u]));
+                    mx = __int2float_rn(max(max(mi[0], mi[1]), max(mi[2], mi[3])));
+                } else {
+                    float mf[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) mf[u] = __uint_as_float(s[u]);
+#pragma unroll
+                    for (int c = 4; c < T - 4; c += 8) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            mf[u] = fmax3(mf[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) mf[u] = fmaxf(mf[u], __uint_as_float(s[T - 4 + u]));
+                    mx = fmaxf(fmaxf(mf[0], mf[1]), fmaxf(mf[2], mf[3]));
                 }
                 // shared online-softmax state (Sec. 3.1) in the log2 domain
                 const float m_tile = mx * a;
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long st2 = clock64() + (__float_as_int(m_tile) & 0);
+#endif
                 const bool grow = m_tile > m_run + kTau;
                 float alpha = 1.f;
                 if (grow) {
                     alpha = fast_exp2(m_run - m_tile);
                     m_run = m_tile;
                 }
-                float sum = 0.f;
-                // P = 2^(a*raw - m), rounded to FP16 and packed two per word into s[0 .. T/2)
+                // P = 2^(a*raw - m), rounded to FP16 and packed two per word into s[0 .. T/2).
+                // Two elements per packed FP32x2 instruction; four independent partial sums.
+                float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+                const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
+                // Work in blocks of 16 columns, one instruction kind at a time, so that the 8 packed
+                // operations of a stage are independent and the special-function unit stays fed.
+                if (int8_route && !diag) {
+                    // int -> float without the conversion unit: bits(1.5*2^23) + i is the float
+                    // 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D), minus 1.5*2^23 is exact.
+                    const float2 magic = make_float2(-12582912.f, -12582912.f);
 #pragma unroll
-                for (int c = 0; c < T; c += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), a, -m_run));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), a, -m_run));
-                    sum += p0 + p1;
-                    const __half2 h = __floats2half2_rn(p0, p1);
-                    s[c >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                    for (int blk = 0; blk < T / 16; ++blk) {
+                        float2 x[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            x[u] = make_float2(__uint_as_float(s[blk * 16 + 2 * u] + 0x4B400000u),
+                                               __uint_as_float(s[blk * 16 + 2 * u + 1] + 0x4B400000u));
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) x[u] = __fadd2_rn(x[u], magic);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) x[u] = __ffma2_rn(x[u], a2, nm2);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) x[u] = make_float2(fast_exp2(x[u].x), fast_exp2(x[u].y));
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) acc[u & 3] = __fadd2_rn(acc[u & 3], x[u]);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) s[blk * 8 + u] = pack_half2(x[u].x, x[u].y);
+                    }
+                } else {
+#pragma unroll
+                    for (int blk = 0; blk < T / 16; ++blk) {
+                        float2 x[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            x[u] = __ffma2_rn(make_float2(__uint_as_float(s[blk * 16 + 2 * u]), __uint_as_float(s[blk * 16 + 2 * u + 1])), a2, nm2);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) x[u] = make_float2(fast_exp2(x[u].x), fast_exp2(x[u].y));
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) acc[u & 3] = __fadd2_rn(acc[u & 3], x[u]);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) s[blk * 8 + u] = pack_half2(x[u].x, x[u].y);
+                    }
                 }
+                const float2 s01 = __fadd2_rn(acc[0], acc[1]), s23 = __fadd2_rn(acc[2], acc[3]);
+                const float sum = (s01.x + s01.y) + (s23.x + s23.y);
                 z = z * alpha + sum;
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long st3 = clock64() + (__float_as_int(z) & 0);
+#endif
 
                 if (j > 0 && __any_sync(0xffffffffu, grow)) {
                     // O~ *= alpha.  PV of tile j-1 has retired: it was issued before the QK^T
@@ -497,8 +635,18 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t));
+#ifdef TILEMIX_PHASE_TIMERS
+                if ((threadIdx.x & 127) == 0) {
+                    const long long st4 = clock64();
+                    TM_TIMER_ADD(40, st1 - st0); TM_TIMER_ADD(41, st2 - st1); TM_TIMER_ADD(42, st3 - st2);
+                    TM_TIMER_ADD(43, st4 - st3); TM_TIMER_ADD(44, 1);
+                }
+#endif
             }
 
+#ifdef TILEMIX_PHASE_TIMERS
+            if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(33 + t, clock64() - loop_c0);
+#endif
             if (ok) {
                 ok = wait_bar(cx, bar_o(t), 0, role, m_t + 1, kBarO);
                 ok = __all_sync(0xffffffffu, ok);
@@ -533,6 +681,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     }
 
     // ---- teardown -----------------------------------------------------------------------
+#ifdef TILEMIX_PHASE_TIMERS
+    if (threadIdx.x == 0) {
+        TM_TIMER_ADD(32, clock64() - cta_c0);
+        TM_TIMER_ADD(35, 1);
+        TM_TIMER_ADD(36, nkv);
+    }
+#endif
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) {
@@ -610,7 +765,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     if (dbg != nullptr && dbg->n_tiles > 0) {
         prm.dbg_tiles = dbg->tiles; prm.dbg_n = dbg->n_tiles; prm.dbg_raw = dbg->raw; prm.dbg_kind = dbg->kind;
     }
-    cudaError_t e = cudaMemsetAsync(workspace, 0, 16, stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceClearBytes, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
     e = cudaFuncSetAttribute(attention_kernel<D, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
     if (e != cudaSuccess) return static_cast<int>(e);
