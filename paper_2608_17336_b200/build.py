@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.path.join(HERE, "libtilemix.so")
+LIB = os.environ.get("TILEMIX_LIB", os.path.join(HERE, "libtilemix.so"))
 SOURCES = ["api.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu"]
 HEADERS = ["common.cuh", "ptx_sm100.cuh"]
 

@@ -144,7 +144,7 @@ int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {
 size_t tilemix_workspace_size(const tilemix_problem_t* p) {
     Geometry g;
     if (resolve(p, &g)) return 0;
-    return 1024;   // status record (16 bytes) + optional phase timers
+    return 4096;   // status record (16 bytes) + optional phase timers / trace
 }
 
 size_t tilemix_scratch_bytes(const tilemix_problem_t* p) {
@@ -173,7 +173,7 @@ Arena arena_layout(const Geometry& g) {
     a.ks = put(4u * static_cast<size_t>(g.B) * g.Hk * ceil_div(g.L, g.blk_k));
     a.route = put(static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.T_mask);
     a.words = put(4u * static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.W);
-    a.work = put(1024);
+    a.work = put(4096);
     a.total = off;
     return a;
 }
@@ -218,7 +218,7 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
     if ((rc = tilemix_attention_fwd(&dense, base + a.q, base + a.k, base + a.v, reinterpret_cast<int8_t*>(base + a.q8),
                                     reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
                                     reinterpret_cast<float*>(base + a.ks), reinterpret_cast<uint32_t*>(base + a.words),
-                                    base + a.o, nullptr, base + a.work, 1024, nullptr, stream)))
+                                    base + a.o, nullptr, base + a.work, 4096, nullptr, stream)))
         return rc;
     if ((e = cudaMemcpyAsync(out_host, base + a.o, nq * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return e;
     return TILEMIX_OK;

@@ -19,6 +19,7 @@
 // roles poll, drains what is in flight and returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
+#include <limits.h>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
@@ -30,9 +31,10 @@ namespace {
 constexpr int kWarpsPerGroup = 4;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
+constexpr int kRegsSoftmax = 200, kRegsOther = 104;   // 2*128*200 + 128*104 = 64512 <= the 64K file, with slack   // register split made with setmaxnreg
 constexpr int kRing = 8;
-constexpr int kWorkspaceClearBytes = 1024;  // status record + optional phase timers
+constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
 constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -161,6 +163,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// 2^x for x <= ~kTau on the FMA pipe (no special-function unit): x = n + f with n = round(x),
+// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.5e-5, below the FP16 rounding of P);
+// 2^n by adding n to the exponent field.  Inputs are clamped to >= -126.
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+    const float2 magic = make_float2(12582912.f, 12582912.f);       // 1.5 * 2^23
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 r = __fadd2_rn(x, magic);                           // low mantissa bits = round(x)
+    const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
+    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+    float2 p = __ffma2_rn(f, make_float2(0.055171649903059006f, 0.055171649903059006f),
+                          make_float2(0.2426111251115799f, 0.2426111251115799f));
+    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+    p = __ffma2_rn(p, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
+    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
+    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
+    return p;
+}
+
+// Every kPolyEvery-th pair of an interior tile takes the polynomial instead of the special-function
+// unit (0 = none), so that both pipes work on a tile at the same time.
+#ifndef TILEMIX_POLY_EVERY
+#define TILEMIX_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = TILEMIX_POLY_EVERY;
+
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -171,6 +199,74 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// One interior score tile in one pass: raw accumulators in tensor memory at t_s -> P = 2^(a*raw - m)
+// rounded to FP16 and packed two per word into p2, the FP32 row sum of P and the row maximum of the
+// raw values.  The 32-column chunks are double-buffered (the next one is in flight while this one is
+// processed), and the per-pair work is software-pipelined in program order -- exponentials of pair
+// k, conversion of pair k + kD1, sum and packing of pair k - (kD2 - kD1) -- because a warp issues in
+// order: the special-function unit takes 16 clocks per pair and the other ~7 instructions of a pair
+// fit in its shadow only if they belong to other pairs.
+template <int T, bool INT8>
+__device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, float a, float m_run, uint32_t (&p2)[T / 2],
+                                                  float& sum, float& mx) {
+    // Pipeline depth in pairs: pair k is read (and, INT8, re-biased) in iteration k, made a float in
+    // k + 1, scaled in k + 2, exponentiated in k + kE and summed / packed in k + kS.  No instruction
+    // uses a result produced in its own iteration.
+    constexpr int NP = T / 2, kE = 3, kS = 7;
+    const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
+    const float2 unbias = make_float2(-12582912.f, -12582912.f);
+    float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+    int mi[4] = {INT_MIN, INT_MIN, INT_MIN, INT_MIN};
+    float mf[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    float2 xb[4], tb[4], eb[8];       // rings: biased / float raw values, scaled values, exponentials
+    uint32_t buf[2][32];
+    ptx::tmem_ld32(t_s, buf[0]);
+#pragma unroll
+    for (int i = 0; i < NP + kS; ++i) {
+        if (i >= kE && i - kE < NP) {                         // exponentials of pair i - kE
+            const int k = i - kE;
+            if (kPolyEvery > 0 && (k % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1)
+                eb[k & 7] = exp2_poly2(tb[k & 3]);
+            else
+                eb[k & 7] = make_float2(fast_exp2(tb[k & 3].x), fast_exp2(tb[k & 3].y));
+        }
+        if (i >= 2 && i - 2 < NP) {                           // a*raw - m of pair i - 2
+            const int k = i - 2;
+            tb[k & 3] = __ffma2_rn(xb[k & 3], a2, nm2);
+        }
+        if (INT8 && i >= 1 && i - 1 < NP) {                   // remove the bias of pair i - 1 (exact)
+            const int k = i - 1;
+            xb[k & 3] = __fadd2_rn(xb[k & 3], unbias);
+        }
+        if (i < NP) {                                         // read pair i
+            const int c = i / 16, e = (i % 16) * 2;
+            if (e == 0) {
+                ptx::tmem_wait_ld_dep(buf[c & 1]);
+                if (c + 1 < T / 32) ptx::tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1) & 1]);
+            }
+            const uint32_t r0 = buf[c & 1][e], r1 = buf[c & 1][e + 1];
+            if (INT8) {
+                // int -> float without the conversion unit: bits(1.5*2^23) + i is the float
+                // 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D); subtracting 1.5*2^23 is exact.
+                mi[i & 3] = __vimax3_s32(mi[i & 3], static_cast<int>(r0), static_cast<int>(r1));
+                xb[i & 3] = make_float2(__uint_as_float(r0 + 0x4B400000u), __uint_as_float(r1 + 0x4B400000u));
+            } else {
+                mf[i & 3] = fmax3(mf[i & 3], __uint_as_float(r0), __uint_as_float(r1));
+                xb[i & 3] = make_float2(__uint_as_float(r0), __uint_as_float(r1));
+            }
+        }
+        if (i >= kS) {                                        // row sum and FP16 packing of pair i - kS
+            const int k = i - kS;
+            acc[k & 3] = __fadd2_rn(acc[k & 3], eb[k & 7]);
+            p2[k] = pack_half2(eb[k & 7].x, eb[k & 7].y);
+        }
+    }
+    mx = INT8 ? __int2float_rn(max(max(mi[0], mi[1]), max(mi[2], mi[3])))
+              : fmaxf(fmaxf(mf[0], mf[1]), fmaxf(mf[2], mf[3]));
+    const float2 s01 = __fadd2_rn(acc[0], acc[1]), s23 = __fadd2_rn(acc[2], acc[3]);
+    sum = (s01.x + s01.y) + (s23.x + s23.y);
 }
 
 template <int D, int T>
@@ -265,8 +361,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const uint32_t tmem_base = misc[0];
     auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
-    if (warp == kProducerWarp) {
+    if (warp >= kMmaWarp + 1) {
+        ptx::setmaxnreg_dec<kRegsOther>();   // idle warps of the third warpgroup
+    } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer
+        ptx::setmaxnreg_dec<kRegsOther>();
         if (lane == 0) {
             ptx::tma_prefetch_desc(&tm_q16);
             ptx::tma_prefetch_desc(&tm_k16);
@@ -322,6 +421,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         }
     } else if (warp == kMmaWarp) {
         // ================================================================ MMA issuer
+        ptx::setmaxnreg_dec<kRegsOther>();
         if (lane == 0) {
             constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, C::kM, T);
             constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, C::kM, T);
@@ -445,6 +545,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         }
     } else {
         // ================================================================ softmax groups
+        ptx::setmaxnreg_inc<kRegsSoftmax>();
         const int t = warp / kWarpsPerGroup;
         const int m_t = t ? mB : mA;
         if (t == 0 || hasB) {
@@ -464,13 +565,15 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 #ifdef TILEMIX_PHASE_TIMERS
             const long long loop_c0 = clock64();
 #endif
+            float dk_next = prm.has_int8 ? dk_row[0] : 0.f;
             for (int j = 0; j <= m_t; ++j) {
                 const uint32_t int8_route = (sched(j) >> t) & 1u;
                 float a = prm.scale_log2;
                 if (int8_route) {
-                    a *= dq * dk_row[j];
+                    a *= dq * dk_next;
                     if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                 }
+                if (prm.has_int8 && j < m_t) dk_next = dk_row[j + 1];   // next tile's scale, ahead of its use
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long sw0 = clock64();
 #endif
@@ -483,134 +586,86 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 ptx::tc_fence_after_sync();
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st0 = clock64();
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && j >= 8 && j < 8 + 48)
+                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2] = st0;
 #endif
 
-                uint32_t s[T];
-#pragma unroll
-                for (int c = 0; c < T / 32; ++c)
-                    ptx::tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-                ptx::tmem_wait_ld();
+                // ---- shared online-softmax state (Sec. 3.1), log2 domain --------------------------
+                // P = 2^(a*raw - m) is rounded to FP16 and packed two per word into p2[0 .. T/2).
+                // The running maximum m is lazy: it moves only when a tile exceeds it by more than
+                // kTau.  So an interior tile is done in ONE pass with the current m, 32 columns at a
+                // time with the next 32 already in flight from tensor memory, while its row maximum is
+                // tracked on the side; only if some row of the warp does exceed m + kTau (rare after
+                // the first tiles) the tile is re-read and redone in the generic two-pass form.
+                const bool diag = (j == m_t);
+                bool redo = diag || j == 0 || prm.dbg_n > 0;
+                float alpha = 1.f, sum = 0.f;
+                bool grow = false;
+                uint32_t p2[T / 2];
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st1 = clock64();
 #endif
-
-                if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
-                    int idx = -1;
-                    if (lane == 0) {
-                        for (int e = 0; e < prm.dbg_n; ++e) {
-                            const int32_t* q = prm.dbg_tiles + 4 * e;
-                            if (q[0] == b && q[1] == hq && q[2] == m_t && q[3] == j) { idx = e; break; }
+                if (!redo) {
+                    float mx;
+                    if (int8_route) softmax_tile_fast<T, true>(t_s, a, m_run, p2, sum, mx);
+                    else softmax_tile_fast<T, false>(t_s, a, m_run, p2, sum, mx);
+                    redo = __any_sync(0xffffffffu, mx * a > m_run + kTau);
+                }
+#ifdef TILEMIX_PHASE_TIMERS
+                const long long st2 = clock64() + (__float_as_int(sum) & 0);
+#endif
+                if (redo) {
+                    // Generic two-pass form: first and diagonal tiles, tiles that move the maximum, and
+                    // every tile in debug mode.  The raw accumulators are (still) in tensor memory.
+                    uint32_t s[T];
+#pragma unroll
+                    for (int c = 0; c < T / 32; ++c)
+                        ptx::tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+                    ptx::tmem_wait_ld();
+                    if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
+                        int idx = -1;
+                        if (lane == 0) {
+                            for (int e = 0; e < prm.dbg_n; ++e) {
+                                const int32_t* q = prm.dbg_tiles + 4 * e;
+                                if (q[0] == b && q[1] == hq && q[2] == m_t && q[3] == j) { idx = e; break; }
+                            }
+                        }
+                        idx = __shfl_sync(0xffffffffu, idx, 0);
+                        if (idx >= 0 && row < T) {
+                            int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + row) * T;
+#pragma unroll
+                            for (int c = 0; c < T; c += 4)
+                                *reinterpret_cast<uint4*>(dst + c) = make_uint4(s[c], s[c + 1], s[c + 2], s[c + 3]);
+                            if (row == 0) prm.dbg_kind[idx] = static_cast<uint8_t>(int8_route);
                         }
                     }
-                    idx = __shfl_sync(0xffffffffu, idx, 0);
-                    if (idx >= 0 && row < T) {
-                        int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + row) * T;
-#pragma unroll
-                        for (int c = 0; c < T; c += 4)
-                            *reinterpret_cast<uint4*>(dst + c) = make_uint4(s[c], s[c + 1], s[c + 2], s[c + 3]);
-                        if (row == 0) prm.dbg_kind[idx] = static_cast<uint8_t>(int8_route);
-                    }
-                }
-
-                // Row maximum of the raw accumulators.  The scale a is >= 0, so max(a*raw) =
-                // a*max(raw); for INT8 tiles the maximum is taken on the integers.
-                const bool diag = (j == m_t);
-                float mx;
-                if (diag) {
-                    // Diagonal tile (one per row of tiles): generic path.  Convert to FP32 and
-                    // apply causal legality (App. B: enforced kernel-side, independent of R).
-                    mx = -INFINITY;
+                    // Common FP32 score domain (App. C), causal legality on the diagonal tile (App. B:
+                    // enforced kernel-side, independent of R), row maximum, then the exponentials.
+                    float mx = -INFINITY;
 #pragma unroll
                     for (int c = 0; c < T; ++c) {
                         float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
-                        if (c > row) v = -INFINITY;
+                        if (diag && c > row) v = -INFINITY;
                         s[c] = __float_as_uint(v);
                         mx = fmaxf(mx, v);
                     }
-                } else if (int8_route) {
-                    int mi[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) mi[u] = static_cast<int>(s[u]);
-#pragma unroll
-                    for (int c = 4; c < T - 4; c += 8) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            mi[u] = __vimax3_s32(mi[u], static_cast<int>(s[c + 2 * u]), static_cast<int>(s[c + 2 * u + 1]));
+                    const float m_tile = mx * a;     // a >= 0, so max(a*raw) = a*max(raw)
+                    grow = m_tile > m_run + kTau;
+                    if (grow) {
+                        alpha = fast_exp2(m_run - m_tile);
+                        m_run = m_tile;
                     }
-                    // (T - 4) % 8 == 4: the last four columns
+                    const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
+                    float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) mi[u] = max(mi[u], static_cast<int>(s[T - 4 + u]));
-                    mx = __int2float_rn(max(max(mi[0], mi[1]), max(mi[2], mi[3])));
-                } else {
-                    float mf[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) mf[u] = __uint_as_float(s[u]);
-#pragma unroll
-                    for (int c = 4; c < T - 4; c += 8) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            mf[u] = fmax3(mf[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
+                    for (int c = 0; c < T; c += 2) {
+                        const float2 t2 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), a2, nm2);
+                        const float2 pp = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
+                        acc = __fadd2_rn(acc, pp);
+                        p2[c >> 1] = pack_half2(pp.x, pp.y);
                     }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) mf[u] = fmaxf(mf[u], __uint_as_float(s[T - 4 + u]));
-                    mx = fmaxf(fmaxf(mf[0], mf[1]), fmaxf(mf[2], mf[3]));
+                    sum = acc.x + acc.y;
                 }
-                // shared online-softmax state (Sec. 3.1) in the log2 domain
-                const float m_tile = mx * a;
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long st2 = clock64() + (__float_as_int(m_tile) & 0);
-#endif
-                const bool grow = m_tile > m_run + kTau;
-                float alpha = 1.f;
-                if (grow) {
-                    alpha = fast_exp2(m_run - m_tile);
-                    m_run = m_tile;
-                }
-                // P = 2^(a*raw - m), rounded to FP16 and packed two per word into s[0 .. T/2).
-                // Two elements per packed FP32x2 instruction; four independent partial sums.
-                float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-                const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
-                // Work in blocks of 16 columns, one instruction kind at a time, so that the 8 packed
-                // operations of a stage are independent and the special-function unit stays fed.
-                if (int8_route && !diag) {
-                    // int -> float without the conversion unit: bits(1.5*2^23) + i is the float
-                    // 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D), minus 1.5*2^23 is exact.
-                    const float2 magic = make_float2(-12582912.f, -12582912.f);
-#pragma unroll
-                    for (int blk = 0; blk < T / 16; ++blk) {
-                        float2 x[8];
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            x[u] = make_float2(__uint_as_float(s[blk * 16 + 2 * u] + 0x4B400000u),
-                                               __uint_as_float(s[blk * 16 + 2 * u + 1] + 0x4B400000u));
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) x[u] = __fadd2_rn(x[u], magic);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) x[u] = __ffma2_rn(x[u], a2, nm2);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) x[u] = make_float2(fast_exp2(x[u].x), fast_exp2(x[u].y));
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) acc[u & 3] = __fadd2_rn(acc[u & 3], x[u]);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) s[blk * 8 + u] = pack_half2(x[u].x, x[u].y);
-                    }
-                } else {
-#pragma unroll
-                    for (int blk = 0; blk < T / 16; ++blk) {
-                        float2 x[8];
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            x[u] = __ffma2_rn(make_float2(__uint_as_float(s[blk * 16 + 2 * u]), __uint_as_float(s[blk * 16 + 2 * u + 1])), a2, nm2);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) x[u] = make_float2(fast_exp2(x[u].x), fast_exp2(x[u].y));
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) acc[u & 3] = __fadd2_rn(acc[u & 3], x[u]);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) s[blk * 8 + u] = pack_half2(x[u].x, x[u].y);
-                    }
-                }
-                const float2 s01 = __fadd2_rn(acc[0], acc[1]), s23 = __fadd2_rn(acc[2], acc[3]);
-                const float sum = (s01.x + s01.y) + (s23.x + s23.y);
                 z = z * alpha + sum;
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st3 = clock64() + (__float_as_int(z) & 0);
@@ -631,13 +686,15 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 }
 #pragma unroll
                 for (int c = 0; c < T / 64; ++c)
-                    ptx::tmem_st32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+                    ptx::tmem_st32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p2[c * 32]));
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t));
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) {
                     const long long st4 = clock64();
+                    if (blockIdx.x == 5 && j >= 8 && j < 8 + 48)
+                        reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2 + 1] = st4;
                     TM_TIMER_ADD(40, st1 - st0); TM_TIMER_ADD(41, st2 - st1); TM_TIMER_ADD(42, st3 - st2);
                     TM_TIMER_ADD(43, st4 - st3); TM_TIMER_ADD(44, 1);
                 }

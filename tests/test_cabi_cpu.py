@@ -61,7 +61,7 @@ def test_host_side_validation_without_gpu(lib):
     odd.q_stride[0], odd.q_stride[1], odd.q_stride[2] = 2 * 1024 * 132, 1024 * 132, 132
     assert lib.tilemix_quantize_qk(ctypes.byref(odd), *_args(6), null) == b.ERR_ALIGN
     # attention: unsupported tile / head_dim / quant block, missing INT8 operands, small workspace
-    att = lambda p, ws=1024, q8=0x1000: lib.tilemix_attention_fwd(
+    att = lambda p, ws=4096, q8=0x1000: lib.tilemix_attention_fwd(
         ctypes.byref(p), *_args(3), ctypes.c_void_p(q8) if q8 else None, *_args(5), None, ctypes.c_void_p(0x1000), ws, None, None)
     assert att(b.problem(1, 2, 2, 1024, 128, 64, 64)) == b.ERR_UNSUPPORTED
     assert att(b.problem(1, 2, 2, 1024, 96, 128, 128)) == b.ERR_UNSUPPORTED
@@ -70,7 +70,7 @@ def test_host_side_validation_without_gpu(lib):
     assert att(good, q8=0) == b.ERR_NULL
     assert att(good, q8=0x1001) == b.ERR_ALIGN
     dbg = b.DebugStruct(None, 3, None, None)
-    assert lib.tilemix_attention_fwd(ctypes.byref(good), *_args(9), None, ctypes.c_void_p(0x1000), 1024,
+    assert lib.tilemix_attention_fwd(ctypes.byref(good), *_args(9), None, ctypes.c_void_p(0x1000), 4096,
                                      ctypes.byref(dbg), None) == b.ERR_NULL
     assert lib.tilemix_launch_count() == 0
 
