@@ -19,10 +19,10 @@
 // roles poll, drains what is in flight and returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
-#include <limits.h>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "softmax_tile.cuh"
 
 namespace tilemix {
 
@@ -156,118 +156,6 @@ struct Ring {
     __device__ __forceinline__ uint32_t phase(uint32_t s) const { return (phases >> s) & 1u; }
     __device__ __forceinline__ void flip(uint32_t s) { phases ^= 1u << s; }
 };
-
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// 2^x for x <= ~kTau on the FMA pipe (no special-function unit): x = n + f with n = round(x),
-// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.5e-5, below the FP16 rounding of P);
-// 2^n by adding n to the exponent field.  Inputs are clamped to >= -126.
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    const float2 magic = make_float2(12582912.f, 12582912.f);       // 1.5 * 2^23
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 r = __fadd2_rn(x, magic);                           // low mantissa bits = round(x)
-    const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p = __ffma2_rn(f, make_float2(0.055171649903059006f, 0.055171649903059006f),
-                          make_float2(0.2426111251115799f, 0.2426111251115799f));
-    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
-    p = __ffma2_rn(p, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
-    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
-    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
-    return p;
-}
-
-// Every kPolyEvery-th pair of an interior tile takes the polynomial instead of the special-function
-// unit (0 = none), so that both pipes work on a tile at the same time.
-#ifndef TILEMIX_POLY_EVERY
-#define TILEMIX_POLY_EVERY 0
-#endif
-constexpr int kPolyEvery = TILEMIX_POLY_EVERY;
-
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-// One interior score tile in one pass: raw accumulators in tensor memory at t_s -> P = 2^(a*raw - m)
-// rounded to FP16 and packed two per word into p2, the FP32 row sum of P and the row maximum of the
-// raw values.  The 32-column chunks are double-buffered (the next one is in flight while this one is
-// processed), and the per-pair work is software-pipelined in program order -- exponentials of pair
-// k, conversion of pair k + kD1, sum and packing of pair k - (kD2 - kD1) -- because a warp issues in
-// order: the special-function unit takes 16 clocks per pair and the other ~7 instructions of a pair
-// fit in its shadow only if they belong to other pairs.
-template <int T, bool INT8>
-__device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, float a, float m_run, uint32_t (&p2)[T / 2],
-                                                  float& sum, float& mx) {
-    // Pipeline depth in pairs: pair k is read (and, INT8, re-biased) in iteration k, made a float in
-    // k + 1, scaled in k + 2, exponentiated in k + kE and summed / packed in k + kS.  No instruction
-    // uses a result produced in its own iteration.
-    constexpr int NP = T / 2, kE = 3, kS = 7;
-    const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
-    const float2 unbias = make_float2(-12582912.f, -12582912.f);
-    float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-    int mi[4] = {INT_MIN, INT_MIN, INT_MIN, INT_MIN};
-    float mf[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    float2 xb[4], tb[4], eb[8];       // rings: biased / float raw values, scaled values, exponentials
-    uint32_t buf[2][32];
-    ptx::tmem_ld32(t_s, buf[0]);
-#pragma unroll
-    for (int i = 0; i < NP + kS; ++i) {
-        if (i >= kE && i - kE < NP) {                         // exponentials of pair i - kE
-            const int k = i - kE;
-            if (kPolyEvery > 0 && (k % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1)
-                eb[k & 7] = exp2_poly2(tb[k & 3]);
-            else
-                eb[k & 7] = make_float2(fast_exp2(tb[k & 3].x), fast_exp2(tb[k & 3].y));
-        }
-        if (i >= 2 && i - 2 < NP) {                           // a*raw - m of pair i - 2
-            const int k = i - 2;
-            tb[k & 3] = __ffma2_rn(xb[k & 3], a2, nm2);
-        }
-        if (INT8 && i >= 1 && i - 1 < NP) {                   // remove the bias of pair i - 1 (exact)
-            const int k = i - 1;
-            xb[k & 3] = __fadd2_rn(xb[k & 3], unbias);
-        }
-        if (i < NP) {                                         // read pair i
-            const int c = i / 16, e = (i % 16) * 2;
-            if (e == 0) {
-                ptx::tmem_wait_ld_dep(buf[c & 1]);
-                if (c + 1 < T / 32) ptx::tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1) & 1]);
-            }
-            const uint32_t r0 = buf[c & 1][e], r1 = buf[c & 1][e + 1];
-            if (INT8) {
-                // int -> float without the conversion unit: bits(1.5*2^23) + i is the float
-                // 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D); subtracting 1.5*2^23 is exact.
-                mi[i & 3] = __vimax3_s32(mi[i & 3], static_cast<int>(r0), static_cast<int>(r1));
-                xb[i & 3] = make_float2(__uint_as_float(r0 + 0x4B400000u), __uint_as_float(r1 + 0x4B400000u));
-            } else {
-                mf[i & 3] = fmax3(mf[i & 3], __uint_as_float(r0), __uint_as_float(r1));
-                xb[i & 3] = make_float2(__uint_as_float(r0), __uint_as_float(r1));
-            }
-        }
-        if (i >= kS) {                                        // row sum and FP16 packing of pair i - kS
-            const int k = i - kS;
-            acc[k & 3] = __fadd2_rn(acc[k & 3], eb[k & 7]);
-            p2[k] = pack_half2(eb[k & 7].x, eb[k & 7].y);
-        }
-    }
-    mx = INT8 ? __int2float_rn(max(max(mi[0], mi[1]), max(mi[2], mi[3])))
-              : fmaxf(fmaxf(mf[0], mf[1]), fmaxf(mf[2], mf[3]));
-    const float2 s01 = __fadd2_rn(acc[0], acc[1]), s23 = __fadd2_rn(acc[2], acc[3]);
-    sum = (s01.x + s01.y) + (s23.x + s23.y);
-}
 
 template <int D, int T>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -586,8 +474,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 ptx::tc_fence_after_sync();
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st0 = clock64();
+#endif
+#ifdef TILEMIX_TRACE
                 if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && j >= 8 && j < 8 + 48)
-                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2] = st0;
+                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2] = clock64();
 #endif
 
                 // ---- shared online-softmax state (Sec. 3.1), log2 domain --------------------------
@@ -690,11 +580,14 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t));
+#ifdef TILEMIX_TRACE
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && j >= 8 && j < 8 + 48)
+                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2 + 1] = clock64();
+#endif
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) {
                     const long long st4 = clock64();
-                    if (blockIdx.x == 5 && j >= 8 && j < 8 + 48)
-                        reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2 + 1] = st4;
+
                     TM_TIMER_ADD(40, st1 - st0); TM_TIMER_ADD(41, st2 - st1); TM_TIMER_ADD(42, st3 - st2);
                     TM_TIMER_ADD(43, st4 - st3); TM_TIMER_ADD(44, 1);
                 }
