@@ -121,6 +121,31 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
                           void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg,
                           void* stream);
 
+/* Same computation as tilemix_attention_fwd for callers that cannot hand it a workspace because
+ * they cannot allocate device memory at all: a process whose whole GPU memory was claimed at
+ * start-up by another allocator or memory pool (any later cudaMalloc fails), or a code path that
+ * must not synchronise the device, which cudaMalloc and cudaFree do.  (The paper has no
+ * counterpart; this is a convenience of this library.)  The workspace is a fixed array of
+ * 4096 bytes inside the library image; every GPU on which the library is used holds its own copy
+ * until the process exits.  This call allocates nothing -- no cudaMalloc, no cudaFree, no
+ * allocating library routine -- and all inputs and outputs are still the caller's.
+ *   - A problem whose tilemix_workspace_size() exceeds 4096 bytes is rejected with
+ *     TILEMIX_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the device address of the array (a host-side query, that
+ *     device must be current); make that first call before any stream capture begins.
+ *   - Every call on a device shares the one array, which keeps what the last call left in it; this
+ *     call clears the status record on `stream` before the kernel.  Two calls that overlap on the
+ *     GPU (different streams, or different host threads on different streams) race on the status
+ *     record: serialise them, or use tilemix_attention_fwd with one workspace per stream.
+ *   workspace_out  nullable; receives the device address of the array, e.g. for tilemix_read_status
+ * All other parameters, the return values and the error behaviour are those of
+ * tilemix_attention_fwd. */
+int tilemix_attention_fwd_noalloc(const tilemix_problem_t* p, const void* q_f16, const void* k_f16,
+                                  const void* v_f16, const int8_t* q_i8, const int8_t* k_i8,
+                                  const float* q_scale, const float* k_scale,
+                                  const uint32_t* mask_words, void* out_f16, float* lse,
+                                  const tilemix_debug_t* dbg, void** workspace_out, void* stream);
+
 /* Whole path on HOST buffers: copies Q, K, V and the routing map to the device arena,
  * quantises, packs, runs the fused kernel and copies O back; everything is enqueued on
  * `stream` in order (use pinned host memory for the copies to be asynchronous).

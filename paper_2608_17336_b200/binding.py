@@ -17,7 +17,8 @@ FORCE_FP16 = 1
 PIN_DIAGONAL_FP16 = 1
 
 EXPORTS = (
-    "tilemix_quantize_qk", "tilemix_pack_routing_mask", "tilemix_attention_fwd", "tilemix_prefill_host",
+    "tilemix_quantize_qk", "tilemix_pack_routing_mask", "tilemix_attention_fwd", "tilemix_attention_fwd_noalloc",
+    "tilemix_prefill_host",
     "tilemix_mask_words_per_row", "tilemix_workspace_size", "tilemix_scratch_bytes", "tilemix_arena_size",
     "tilemix_read_status", "tilemix_status_string", "tilemix_launch_count",
 )
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.tilemix_pack_routing_mask.argtypes = [pp, vp, u32, vp, vp, vp]
         L.tilemix_attention_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t,
                                             ctypes.POINTER(DebugStruct), vp]
+        L.tilemix_attention_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                    ctypes.POINTER(DebugStruct), ctypes.POINTER(vp), vp]
         L.tilemix_prefill_host.argtypes = [pp, vp, vp, vp, vp, u32, vp, vp, ctypes.c_size_t, vp]
         L.tilemix_mask_words_per_row.argtypes = [i32, i32, i32]
         for name in ("tilemix_workspace_size", "tilemix_scratch_bytes", "tilemix_arena_size"):
@@ -174,6 +177,28 @@ def tilemix_attention_fwd(p: ProblemStruct, q, k, v, q8=None, k8=None, q_scale=N
                                      workspace.numel(), ctypes.byref(dbg) if dbg is not None else None, _stream())
     _check(rc, "tilemix_attention_fwd")
     return {"out": out, "lse": lse, "raw": raw, "kind": kind, "workspace": workspace}
+
+
+def tilemix_attention_fwd_noalloc(p: ProblemStruct, q, k, v, q8, k8, q_scale, k_scale, words, out, lse=None):
+    """The fused forward for callers that cannot allocate device memory: every tensor, `out` included,
+    is passed in, and the library's built-in 4096-byte workspace replaces the caller's.  Nothing is
+    allocated here or in the library.  Returns the device address (int) of that workspace; pass it to
+    tilemix_read_status_at to read the status record.  Calls on one device share the workspace, so do
+    not let two of them overlap on the GPU."""
+    pp = _with_strides(p, q=q, k=k, v=v, o=out)
+    ws = ctypes.c_void_p()
+    rc = lib().tilemix_attention_fwd_noalloc(ctypes.byref(pp), _ptr(q), _ptr(k), _ptr(v), _ptr(q8), _ptr(k8),
+                                             _ptr(q_scale), _ptr(k_scale), _ptr(words), _ptr(out), _ptr(lse), None,
+                                             ctypes.byref(ws), _stream())
+    _check(rc, "tilemix_attention_fwd_noalloc")
+    return ws.value
+
+
+def tilemix_read_status_at(workspace_addr: int):
+    """tilemix_read_status on a raw device address (synchronises the current stream)."""
+    rec = (ctypes.c_int32 * 4)()
+    rc = lib().tilemix_read_status(ctypes.c_void_p(workspace_addr), ctypes.byref(rec), _stream())
+    return rc, list(rec)
 
 
 def tilemix_read_status(workspace: torch.Tensor):

@@ -739,3 +739,54 @@ int launch_attention(const Geometry& g, const void* q, const void* k, const void
 }
 
 }  // namespace tilemix
+
+// ---------------------------------------------------------------------------------- no-allocation entry
+// Scratch for callers that cannot allocate device memory: the status/workspace record of
+// tilemix_attention_fwd, held in a fixed array that lives in the library image.
+namespace tilemix {
+namespace {
+
+constexpr size_t kStaticWorkspaceBytes = 4096;
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+constexpr int kMaxDevices = 64;
+std::atomic<void*> g_static_workspace_addr[kMaxDevices];
+
+// Device address of g_static_workspace on the current device.  In host code the array's name is only
+// a handle, not a device address, so the address is asked for once per device (that device current).
+int static_workspace(void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    if (dev < 0 || dev >= kMaxDevices) return TILEMIX_ERR_UNSUPPORTED;
+    void* ptr = g_static_workspace_addr[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
+        e = cudaGetSymbolAddress(&ptr, g_static_workspace);
+        if (e != cudaSuccess) return static_cast<int>(e);
+        if (ptr == nullptr) return static_cast<int>(cudaErrorInvalidSymbol);
+        g_static_workspace_addr[dev].store(ptr, std::memory_order_release);   // same value from any thread
+    }
+    *out = ptr;
+    return TILEMIX_OK;
+}
+
+}  // namespace
+}  // namespace tilemix
+
+extern "C" int tilemix_attention_fwd_noalloc(const tilemix_problem_t* p, const void* q_f16, const void* k_f16,
+                                             const void* v_f16, const int8_t* q_i8, const int8_t* k_i8,
+                                             const float* q_scale, const float* k_scale,
+                                             const uint32_t* mask_words, void* out_f16, float* lse,
+                                             const tilemix_debug_t* dbg, void** workspace_out, void* stream) {
+    using namespace tilemix;
+    if (p == nullptr || !q_f16 || !k_f16 || !v_f16 || !out_f16) return TILEMIX_ERR_NULL;
+    const size_t need = tilemix_workspace_size(p);
+    if (need == 0) return TILEMIX_ERR_SHAPE;
+    if (need > kStaticWorkspaceBytes) return TILEMIX_ERR_WORKSPACE;   // beyond the fixed scratch
+    void* ws = nullptr;
+    const int rc = static_workspace(&ws);
+    if (rc != TILEMIX_OK) return rc;
+    if (workspace_out != nullptr) *workspace_out = ws;
+    return tilemix_attention_fwd(p, q_f16, k_f16, v_f16, q_i8, k_i8, q_scale, k_scale, mask_words, out_f16, lse,
+                                 ws, kStaticWorkspaceBytes, dbg, stream);
+}
