@@ -117,6 +117,25 @@ def oracle_sample(w: synth.Workload, q, k, v, route, budget_pairs: float):
     return dt, int((rows[:, 2] + 1).sum()), len(rows), oracle.num_threads()
 
 
+def rank_workload(w: synth.Workload, rank: int) -> synth.Workload:
+    """Every rank runs its own batch of the same shape: same recipe, rank-dependent seed."""
+    return w.scaled(seed=w.seed + 1000 * rank)
+
+
+def max_over_ranks(values, device, world: int):
+    """Element-wise maximum of per-rank device timings (the job is as slow as its slowest rank)."""
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def job_value(flops_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Whole-job effective TFLOP/s: all ranks' FLOPs over the slowest rank's step time."""
+    return world * flops_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
 def run_reference(args, w, rank, world):
     """--impl reference: the CPU oracle on the host cores, on a bounded sample per step."""
     if rank != 0:
@@ -179,7 +198,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    w_rank = w.scaled(seed=w.seed + 1000 * rank)      # every rank its own batch of the same shape
+    w_rank = rank_workload(w, rank)
 
     q, k, v = synth.make_qkv(w_rank)
     route = synth.make_route(w_rank)
@@ -254,10 +273,7 @@ def main():
         del arena
 
     # ---- max over ranks ----------------------------------------------------------------------------------
-    t = torch.tensor([total_ms, attn_ms, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, attn_ms, e2e_ms = (float(x) for x in t.cpu())
+    total_ms, attn_ms, e2e_ms = max_over_ranks([total_ms, attn_ms, e2e["ms"] if e2e else 0.0], dev, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -265,7 +281,7 @@ def main():
 
     F = effective_flops(w)
     ms_per_step = total_ms / args.steps
-    value = world * F / (ms_per_step * 1e-3) / 1e12
+    value = job_value(F, world, ms_per_step)
     peaks, peak_kind = load_peaks()
     # mask-weighted roofline: T = F_pv/P16 + F_qk*((1-f8)/P16 + f8/P8); f8 = INT8 share of legal tiles.
     # f8 from the realised mask: expand groups to tiles on or below the diagonal
@@ -297,7 +313,7 @@ def main():
                      "attention_ms": attn_ms, "peak_sustained": peak_eff_sus, "frac_sustained": achieved / peak_eff_sus},
     }
     if e2e:
-        line["e2e"] = {"value": world * F / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        line["e2e"] = {"value": job_value(F, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(e2e["h2d"]), "d2h_bytes_per_step": int(e2e["d2h"])}
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
