@@ -30,6 +30,9 @@ from paper_2608_17336_b200 import synth  # noqa: E402
 METRIC = "effective causal-attention TFLOP/s at 1 B200 vs INT8 fraction; % of mixed roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
+# profiles/attention_kernel_cfg3_long32k.md (8-head capture: 324.3 MB, traffic scales with the head count).
+NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 324.3e6 / 8}
 
 
 def effective_flops(w: synth.Workload) -> float:
@@ -307,7 +310,9 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks.summary(),
         "roofline": {"bound": "tensor", "kernel": "attention_kernel", "achieved": achieved, "peak": peak_eff,
-                     "unit": "TFLOP/s", "frac": achieved / peak_eff, "traffic": None,
+                     "unit": "TFLOP/s", "frac": achieved / peak_eff,
+                     "traffic": (NCU_DRAM_BYTES_PER_HEAD[w.name] * w.heads * w.batch if w.name in NCU_DRAM_BYTES_PER_HEAD else None),
+                     "traffic_unit": "bytes per launch (ncu dram read+write, scaled from an 8-head capture)",
                      "peak_source": f"{peak_kind}: bf16 burst {p16} TFLOP/s, INT8 = {INT8_OVER_FP16}x nominal ratio, "
                                     f"mask-weighted with f8={f8:.4f}",
                      "attention_ms": attn_ms, "peak_sustained": peak_eff_sus, "frac_sustained": achieved / peak_eff_sus},
