@@ -178,6 +178,7 @@ def main():
     ap.add_argument("--heads", type=int, default=None, help="override the head count (smaller profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the INT8-fraction sweep of the attention kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tilemix" else args.warmup
 
@@ -320,6 +321,29 @@ def main():
     if e2e:
         line["e2e"] = {"value": job_value(F, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(e2e["h2d"]), "d2h_bytes_per_step": int(e2e["d2h"])}
+    if world == 1 and not args.no_sweep:
+        # the metric's "vs INT8 fraction" axis: same shapes and inputs, attention kernel only
+        q8, k8, qs, ks = tm.tilemix_quantize_qk(p, qd, kd)
+        sweep = []
+        for frac in (0.0, 0.25, 0.5, 0.75, 1.0):
+            ws = w_rank.scaled(int8_fraction=frac, pin_diagonal=False,
+                               routing="zero" if frac == 0.0 else "one" if frac == 1.0 else "row_exact")
+            words_s, _ = tm.tilemix_pack_routing_mask(p, torch.from_numpy(synth.make_route(ws)).to(dev), False)
+            whs = words_s.cpu().numpy().view(np.uint32)
+            f8s = float(((whs[:, :, mm, gg >> 5] >> (gg & 31).astype(np.uint32)) & 1).mean())
+            for _ in range(2):
+                tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words_s, out=out, workspace=work)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s0.record(stream)
+            for _ in range(5):
+                tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words_s, out=out, workspace=work)
+            s1.record(stream)
+            torch.cuda.synchronize()
+            ms = s0.elapsed_time(s1) / 5
+            pk = p16 / (1.0 - f8s * (1.0 - 1.0 / INT8_OVER_FP16) / 2.0)
+            sweep.append({"int8_tiles": round(f8s, 4), "attention_ms": round(ms, 4),
+                          "tflops": round(F / (ms * 1e-3) / 1e12, 1), "frac": round(F / (ms * 1e-3) / 1e12 / pk, 4)})
+        line["int8_sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
         line["cpu_baseline"] = {"value": 4.0 * w.head_dim * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": threads,

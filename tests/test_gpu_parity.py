@@ -146,6 +146,34 @@ def test_attention_batched_mask_per_batch_and_outliers():
     _full_check(_small("batched", batch=2, heads=2, seqlen=512, mask_batch=2, values="outlier_channels", seed=17))
 
 
+@pytest.mark.parametrize("seed,heads,L,G,frac", [(101, 4, 1536, 1, 0.5), (102, 3, 2048, 2, 0.8), (103, 2, 2304, 3, 0.2),
+                                                  (104, 4, 1280, 1, 0.65), (105, 1, 4096, 4, 0.75)])
+def test_attention_fast_path_many_routing_patterns(seed, heads, L, G, frac):
+    """No debug request, so interior tiles take the one-pass path; every row against the oracle.  The mixes
+    make the two query tiles of a CTA disagree on many key tiles (both copies of K staged)."""
+    _full_check(_small(f"mix{seed}", seed=seed, heads=heads, seqlen=L, group=G, int8_fraction=frac), debug=False)
+    _full_check(_small(f"mix64_{seed}", seed=seed, heads=heads, seqlen=L // 2, head_dim=64, tile=64, group=G,
+                       int8_fraction=frac), debug=False)
+
+
+def test_attention_growing_scores_move_the_running_maximum():
+    """Keys whose magnitude grows along the sequence: later tiles keep exceeding the running maximum, so
+    interior tiles are redone with a new maximum and the output accumulator is rescaled many times."""
+    b = _binding()
+    w = _small("ramp", seqlen=2048, heads=2, seed=61, int8_fraction=0.5)
+    q, k, v = synth.make_qkv(w)
+    ramp = torch.linspace(0.25, 6.0, w.seqlen).view(1, 1, -1, 1)
+    k = (k.float() * ramp).half()
+    q = (q.float() * 1.5).half()
+    route = synth.make_route(w)
+    rows = H.all_rows(w)
+    ref = H.run_oracle(w, q, k, v, route, range(w.heads), rows)
+    res = H.run_gpu(w, q, k, v, route)
+    H.check_rows(res["out"], ref["out"], rows)
+    lse = res["lse"].cpu().numpy().astype(np.float64).reshape(-1)
+    assert np.abs(lse - ref["lse"]).max() < 2e-3 * max(1.0, np.abs(ref["lse"]).max())
+
+
 def test_attention_force_fp16_without_int8_operands():
     b = _binding()
     w = _small("force16", routing="zero", seqlen=512)
