@@ -214,7 +214,11 @@ def main():
     stream = torch.cuda.current_stream()
 
     def step(record=None):
+        if record is not None:
+            record[2].record(stream)
         q8, k8, qs, ks = tm.tilemix_quantize_qk(p, qd, kd)
+        if record is not None:
+            record[3].record(stream)
         words, counts = tm.tilemix_pack_routing_mask(p, rd, w.pin_diagonal)
         if record is not None:
             record[0].record(stream)
@@ -239,7 +243,7 @@ def main():
 
     # ---- timed region: K steps, device-timed, inputs (1 GiB+) far larger than L2 ----------------------
     launches0 = tm.tilemix_launch_count()
-    kern_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    kern_ev = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(4)) for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     with ClockSampler(local_rank) as clocks:
@@ -250,7 +254,9 @@ def main():
         sync_all()
     launches = tm.tilemix_launch_count() - launches0
     total_ms = e0.elapsed_time(e1)
-    attn_ms = sum(a.elapsed_time(b) for a, b in kern_ev) / args.steps
+    attn_ms = sum(ev[0].elapsed_time(ev[1]) for ev in kern_ev) / args.steps
+    quant_ms = sum(ev[2].elapsed_time(ev[3]) for ev in kern_ev) / args.steps
+    pack_ms = sum(ev[3].elapsed_time(ev[0]) for ev in kern_ev) / args.steps
     code, rec = tm.tilemix_read_status(work)
     if code != 0:
         raise RuntimeError(f"device status {rec}")
@@ -318,6 +324,13 @@ def main():
                                     f"mask-weighted with f8={f8:.4f}",
                      "attention_ms": attn_ms, "peak_sustained": peak_eff_sus, "frac_sustained": achieved / peak_eff_sus},
     }
+    # the HBM-bound pre-pass: 3 bytes per element of Q and K (2 read, 1 written)
+    quant_bytes = 3.0 * 2 * w.batch * w.heads * w.seqlen * w.head_dim
+    line["other_kernels"] = {
+        "quantize_qk": {"ms": quant_ms, "bound": "hbm", "achieved": quant_bytes / (quant_ms * 1e-3) / 1e9,
+                        "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                        "frac": quant_bytes / (quant_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"])},
+        "pack_routing_mask": {"ms": pack_ms}}
     if e2e:
         line["e2e"] = {"value": job_value(F, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(e2e["h2d"]), "d2h_bytes_per_step": int(e2e["d2h"])}

@@ -19,21 +19,32 @@ __device__ __forceinline__ uint32_t habs2_bits(uint32_t v) { return v & 0x7fff7f
 // bit patterns order like unsigned integers.
 __device__ __forceinline__ uint32_t umax2(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
 
-__device__ __forceinline__ int quant1(float x, float delta) {
+// The definition: IEEE quotient x / delta, rounded to the nearest integer, ties to even.
+__device__ __forceinline__ int quant1_exact(float x, float delta) {
     int q = __float2int_rn(__fdiv_rn(x, delta));
     return max(-127, min(127, q));
 }
 
-__device__ __forceinline__ uint2 quant8(const uint4& v, float delta) {
+// Same result without a division per element.  t = x * fl(1/delta) is within 2.3e-5 of the IEEE
+// quotient (|quotient| <= 127.5), so both round to the same integer unless t lies within 1e-4 of a
+// half-integer; only then is the quotient formed exactly.  The rounding itself is done by adding
+// 1.5 * 2^23 (round-to-nearest-even puts the integer in the low mantissa bits).
+__device__ __forceinline__ uint32_t quant1(float x, float delta, float rdelta) {
+    const float t = x * rdelta;
+    const float y = t + 12582912.f;
+    const float d = fabsf(t - (y - 12582912.f));
+    int q = __float_as_int(y) - 0x4B400000;
+    if (d > 0.4999f) q = quant1_exact(x, delta);
+    return static_cast<uint32_t>(q) & 0xffu;
+}
+
+__device__ __forceinline__ uint2 quant8(const uint4& v, float delta, float rdelta) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     uint32_t o[2] = {0u, 0u};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float lo = __half2float(__ushort_as_half(static_cast<unsigned short>(w[i] & 0xffffu)));
-        const float hi = __half2float(__ushort_as_half(static_cast<unsigned short>(w[i] >> 16)));
-        const uint32_t a = static_cast<uint32_t>(quant1(lo, delta)) & 0xffu;
-        const uint32_t b = static_cast<uint32_t>(quant1(hi, delta)) & 0xffu;
-        o[i >> 1] |= (a | (b << 8)) << ((i & 1) * 16);
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        o[i >> 1] |= (quant1(f.x, delta, rdelta) | (quant1(f.y, delta, rdelta) << 8)) << ((i & 1) * 16);
     }
     return make_uint2(o[0], o[1]);
 }
@@ -86,6 +97,7 @@ quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, i
 
     const float amax_f = __half2float(__ushort_as_half(static_cast<unsigned short>(amax)));
     const float delta = __fdiv_rn(amax_f, 127.0f);
+    const float rdelta = __frcp_rn(delta);
     if (threadIdx.x == 0) scale[static_cast<int64_t>(bh) * n_blk + r] = delta;
 
     if (amax == 0u) {  // zero block: delta = 0, xhat = 0 (no division by zero)
@@ -96,12 +108,12 @@ quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, i
 #pragma unroll
     for (int i = 0; i < MAXV; ++i) {
         const int v = threadIdx.x + i * kThreads;
-        if (v < nvec) *reinterpret_cast<uint2*>(dst + static_cast<int64_t>(v) * 8) = quant8(cache[i], delta);
+        if (v < nvec) *reinterpret_cast<uint2*>(dst + static_cast<int64_t>(v) * 8) = quant8(cache[i], delta, rdelta);
     }
     for (int v = threadIdx.x + MAXV * kThreads; v < nvec; v += kThreads) {
         const int row = v / vec_per_row, c8 = v - row * vec_per_row;
         const uint4 t = __ldg(reinterpret_cast<const uint4*>(src + row * s_tok + c8 * 8));
-        *reinterpret_cast<uint2*>(dst + static_cast<int64_t>(v) * 8) = quant8(t, delta);
+        *reinterpret_cast<uint2*>(dst + static_cast<int64_t>(v) * 8) = quant8(t, delta, rdelta);
     }
 }
 
