@@ -32,16 +32,22 @@ constexpr int kWarpsPerGroup = 4;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
-constexpr int kRegsSoftmax = 200, kRegsOther = 104;   // 2*128*200 + 128*104 = 64512 <= the 64K file, with slack   // register split made with setmaxnreg
+constexpr int kRegsSoftmax = 216, kRegsOther = 72;   // setmaxnreg split: 2*128*216 + 128*72 = 64512 of the 65536 registers
 constexpr int kRing = 8;
 constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
 constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-// Lazy rescale: the running maximum only moves when a tile exceeds it by more than this many
-// powers of two, so P stays <= 2^kTau (representable in FP16) and O is rarely rescaled.
-constexpr float kTau = 8.0f;
+// Lazy rescale.  P = 2^(score - m) is handed to the tensor pipe in FP16, so the running maximum m
+// may lag the true row maximum by up to kTauHard powers of two (P <= 2^15 fits; z and O are FP32).
+// A tile whose rows stay within kTauHard of m is never recomputed.  m is kept kMargin ABOVE the largest
+// score seen (P then tops out at 2^-kMargin, still 18 binades above the smallest FP16 subnormal), so a
+// later score has to beat everything before it by 2^(kTauHard + kMargin) to force a recomputation.
+// When some row of a warp got more than kTauSoft above its m, every row of that warp moves its m
+// *after* the tile (O and z are rescaled before the next one): that restores the headroom without
+// touching probabilities already computed, and one pass over O serves all 32 rows.
+constexpr float kTauSoft = 8.0f, kTauHard = 15.0f, kMargin = 6.0f;
 
 enum Role : int { kRoleSoftmaxA = 0, kRoleSoftmaxB = 1, kRoleProducer = 2, kRoleMma = 3 };
 enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6 };
@@ -447,6 +453,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const float dq = prm.has_int8 ? prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t] : 0.f;
             const float* dk_row = prm.has_int8 ? prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.T_m : nullptr;
             float m_run = -INFINITY, z = 0.f;
+            float m_seen = -INFINITY;     // largest scaled score seen so far (m_run may lag it)
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
 
@@ -492,6 +499,18 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 float alpha = 1.f, sum = 0.f;
                 bool grow = false;
                 uint32_t p2[T / 2];
+                if (__any_sync(0xffffffffu, m_seen > m_run + kTauSoft)) {
+                    // Deferred move of the maximum decided on the previous tile (all rows of the warp):
+                    // z changes scale here, O~ below together with any move this tile itself forces.
+#ifdef TILEMIX_TRACE
+                    if (lane == 0) atomicAdd(&cx.status[21], 1);
+#endif
+                    const float m_new = fmaxf(m_run, m_seen + kMargin);
+                    alpha = fast_exp2(m_run - m_new);   // 1 for rows that are up to date
+                    m_run = m_new;
+                    z *= alpha;
+                    grow = true;
+                }
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st1 = clock64();
 #endif
@@ -499,10 +518,15 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     float mx;
                     if (int8_route) softmax_tile_fast<T, true>(t_s, a, m_run, p2, sum, mx);
                     else softmax_tile_fast<T, false>(t_s, a, m_run, p2, sum, mx);
-                    redo = __any_sync(0xffffffffu, mx * a > m_run + kTau);
+                    const float m_tile = mx * a;
+                    redo = __any_sync(0xffffffffu, m_tile > m_run + kTauHard);   // P would overflow FP16
+                    if (!redo) m_seen = fmaxf(m_seen, m_tile);
                 }
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st2 = clock64() + (__float_as_int(sum) & 0);
+#endif
+#ifdef TILEMIX_TRACE
+                if (lane == 0) { atomicAdd(&cx.status[22], 1); if (redo) atomicAdd(&cx.status[20], 1); }
 #endif
                 if (redo) {
                     // Generic two-pass form: first and diagonal tiles, tiles that move the maximum, and
@@ -540,10 +564,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         mx = fmaxf(mx, v);
                     }
                     const float m_tile = mx * a;     // a >= 0, so max(a*raw) = a*max(raw)
-                    grow = m_tile > m_run + kTau;
-                    if (grow) {
-                        alpha = fast_exp2(m_run - m_tile);
-                        m_run = m_tile;
+                    // generic form: move at once (to the largest score seen, this tile included)
+                    m_seen = fmaxf(m_seen, m_tile);
+                    float a_now = 1.f;
+                    if (m_seen > m_run + kTauSoft) {
+                        a_now = fast_exp2(m_run - (m_seen + kMargin));
+                        m_run = m_seen + kMargin;
+                        grow = true;
                     }
                     const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
                     float2 acc = make_float2(0.f, 0.f);
@@ -555,8 +582,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         p2[c >> 1] = pack_half2(pp.x, pp.y);
                     }
                     sum = acc.x + acc.y;
+                    z *= a_now;
+                    alpha *= a_now;
                 }
-                z = z * alpha + sum;
+                z += sum;
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st3 = clock64() + (__float_as_int(z) & 0);
 #endif
