@@ -156,6 +156,24 @@ def test_attention_fast_path_many_routing_patterns(seed, heads, L, G, frac):
                        int8_fraction=frac), debug=False)
 
 
+@pytest.mark.parametrize("layout", ["band", "global", "aligned_sparse", "bigbird", "sptrans"])
+def test_attention_structured_layouts(layout):
+    """The paper's structured precision layouts at 50 % coverage, packed and run; all rows vs the oracle."""
+    from paper_2608_17336_b200 import policy
+    b = _binding()
+    w = _small(f"layout_{layout}", seqlen=2048, heads=2, group=2, seed=71)
+    geo, R, info = policy.template(w.seqlen, w.tile, w.tile, layout, 0.5, group=w.group)
+    route = policy.broadcast(R, w.heads)
+    q, k, v = synth.make_qkv(w)
+    rows = H.all_rows(w)
+    ref = H.run_oracle(w, q, k, v, route, range(w.heads), rows)
+    res = H.run_gpu(w, q, k, v, route)
+    assert (res["words"].cpu().numpy().view(np.uint32) == ref["words"]).all()
+    cov = ref["counts"][..., 1].sum() / ref["counts"][..., 0].sum()
+    assert abs(cov - info["coverage"]) < 1e-12
+    H.check_rows(res["out"], ref["out"], rows)
+
+
 def test_attention_growing_scores_move_the_running_maximum():
     """Keys whose magnitude grows along the sequence: later tiles keep exceeding the running maximum, so
     interior tiles are redone with a new maximum and the output accumulator is rescaled many times."""
