@@ -165,6 +165,60 @@ def run_reference(args, w, rank, world):
     }))
 
 
+def varlen_leg(tm, w: synth.Workload, dev, peaks) -> dict:
+    """The same step over a packed variable-length batch (no padding): as many tokens as the dense
+    workload, split into sequences of halving length (L/2, L/4, ... and two of the shortest), Bernoulli
+    routing at the workload's INT8 fraction.  Reported beside the headline; not part of `value`."""
+    total = w.batch * w.seqlen
+    lens, rest = [], total
+    while rest > 2 * 256 and len(lens) < 6:
+        lens.append(rest // 2)
+        rest -= lens[-1]
+    lens += [rest // 2, rest - rest // 2]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64).tolist()
+    gen = torch.Generator(device="cpu").manual_seed(w.seed + 7)
+    qkv = [torch.randn((total, w.heads, w.head_dim), generator=gen).half().to(dev) for _ in range(3)]
+    p = tm.problem(1, w.heads, w.heads, total, w.head_dim, w.tile, w.tile, w.group)
+    vl = tm.Varlen(cu)
+    c = tm.tilemix_varlen_counts(p, vl)
+    rng = np.random.default_rng(w.seed + 8)
+    route = torch.from_numpy((rng.random((w.heads, c["sum_T_m"], c["T_mask_max"])) < w.int8_fraction)
+                             .astype(np.uint8)).to(dev)
+    work = torch.empty(tm.tilemix_varlen_workspace_size(p, vl), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(qkv[0])
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        q8, k8, qs, ks = tm.tilemix_quantize_qk_varlen(p, vl, qkv[0], qkv[1], workspace=work)
+        words, _ = tm.tilemix_pack_routing_mask_varlen(p, vl, route, w.pin_diagonal, workspace=work)
+        if ev:
+            ev[0].record(stream)
+        tm.tilemix_attention_fwd_varlen(p, vl, *qkv, q8, k8, qs, ks, words, out=out, workspace=work)
+        if ev:
+            ev[1].record(stream)
+
+    for _ in range(3):
+        step()
+    n = 5
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for i in range(n):
+        step(evs[i])
+    t1.record(stream)
+    torch.cuda.synchronize()
+    code, rec = tm.tilemix_read_status(work)
+    if code != 0:
+        raise RuntimeError(f"device status {rec}")
+    flops = sum(4.0 * w.heads * float(L) ** 2 * w.head_dim / 2.0 for L in lens)
+    step_ms = t0.elapsed_time(t1) / n
+    attn_ms = sum(a.elapsed_time(b) for a, b in evs) / n
+    return {"seqlens": lens, "tokens": total, "ms_per_step": step_ms, "attention_ms": attn_ms,
+            "value": flops / (step_ms * 1e-3) / 1e12, "attention_tflops": flops / (attn_ms * 1e-3) / 1e12,
+            "unit": "TFLOP/s"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -179,6 +233,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the INT8-fraction sweep of the attention kernel")
+    ap.add_argument("--no-varlen", action="store_true", help="skip the variable-length (packed batch) measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tilemix" else args.warmup
 
@@ -357,6 +412,8 @@ def main():
             sweep.append({"int8_tiles": round(f8s, 4), "attention_ms": round(ms, 4),
                           "tflops": round(F / (ms * 1e-3) / 1e12, 1), "frac": round(F / (ms * 1e-3) / 1e12 / pk, 4)})
         line["int8_sweep"] = sweep
+    if world == 1 and not args.no_varlen and w.tile == 128:
+        line["varlen"] = varlen_leg(tm, w, dev, peaks)
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
         line["cpu_baseline"] = {"value": 4.0 * w.head_dim * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": threads,

@@ -156,6 +156,68 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
                          const void* v_host, const uint8_t* route_host, uint32_t pack_flags,
                          void* out_host, void* arena, size_t arena_bytes, void* stream);
 
+/* ---- variable-length batches (Sec. 4.1, "grouped-query attention and variable-length batching";
+ * App. C, scale shapes for variable-length batches) -------------------------------------------
+ * n_seqs sequences are packed back to back along the token axis with no padding.  Sequence s
+ * owns tokens [cu_seqlens[s], cu_seqlens[s+1]) and is an independent causal attention problem
+ * with its own tiles: T_m(s) = ceil(L_s/tile_m) query-tile rows, blocks of the quantiser that
+ * restart at the sequence's first token, and its own mask rows.  Prefix sums over the sequences
+ * (built by the library from cu_seqlens) place each sequence's tile rows and scale blocks:
+ *   tile_off[s] = sum_{t<s} ceil(L_t/tile_m),  blkq_off / blkk_off likewise with the quantiser
+ *   block sizes.
+ * The problem struct describes the packed batch: batch = 1, seqlen = total tokens
+ * (= cu_seqlens[n_seqs]), mask_batch = 1.  An all-zero stride triple means the flattened
+ * token-major layout [total, H, d] (head stride d, token stride H*d); any other layout is given
+ * by explicit strides (the batch stride is ignored).  Layouts of the derived buffers:
+ *   q_i8, k_i8   INT8 [H, total, d] (head-major, dense)
+ *   q_scale      FP32 [sum_s ceil(L_s/blk_q), Hq]    (block-major, as in App. C)
+ *   k_scale      FP32 [sum_s ceil(L_s/blk_k), Hk]
+ *   route        uint8 [Hk, sum_s T_m(s), T_mask_max], T_mask_max = ceil(max_seqlen/(G*tile_n));
+ *                row tile_off[s]+m is query-tile row m of sequence s; entries beyond the
+ *                sequence's own T_mask(s) are ignored
+ *   mask_words   uint32 [Hk, sum_s T_m(s), W], W = ceil(T_mask_max/32)
+ *   lse          FP32 [Hq, total]
+ * Zero-length sequences are allowed and produce nothing. */
+typedef struct tilemix_varlen {
+    int32_t n_seqs;            /* >= 1                                                         */
+    int32_t max_seqlen;        /* 0 = take the longest sequence of cu_seqlens; otherwise it must
+                                  be >= the longest sequence (fixes T_mask_max and W)          */
+    const int32_t* cu_seqlens; /* HOST pointer, n_seqs + 1 entries, non-decreasing,
+                                  cu_seqlens[0] = 0, cu_seqlens[n_seqs] = p->seqlen; read
+                                  before the call returns                                      */
+} tilemix_varlen_t;
+
+/* Derived sizes of a variable-length batch, out = {total tokens, sum T_m, sum blocks of Q,
+ * sum blocks of K, T_mask_max, W, longest sequence}.  Returns TILEMIX_OK or a negative error. */
+int tilemix_varlen_counts(const tilemix_problem_t* p, const tilemix_varlen_t* vl, int64_t out[7]);
+/* Bytes of `workspace` the three calls below need (0 on invalid arguments): the 4096-byte
+ * status area of tilemix_attention_fwd followed by the prefix-sum tables and the attention
+ * kernel's work list (two int32 per pair of query tiles).  Every call copies
+ * the tables into its workspace on `stream`, so one workspace may serve all three calls in
+ * stream order, and the tables of the last call stay there. */
+size_t tilemix_varlen_workspace_size(const tilemix_problem_t* p, const tilemix_varlen_t* vl);
+/* tilemix_quantize_qk over a variable-length batch: blocks never cross a sequence boundary;
+ * the tail block of every sequence takes its maximum over the rows that exist. */
+int tilemix_quantize_qk_varlen(const tilemix_problem_t* p, const tilemix_varlen_t* vl,
+                               const void* q_f16, const void* k_f16, int8_t* q_i8, int8_t* k_i8,
+                               float* q_scale, float* k_scale, void* workspace,
+                               size_t workspace_bytes, void* stream);
+/* tilemix_pack_routing_mask over a variable-length batch; legality of a group is judged with
+ * the length of the row's own sequence.  counts: nullable uint64 [Hk, 2]. */
+int tilemix_pack_routing_mask_varlen(const tilemix_problem_t* p, const tilemix_varlen_t* vl,
+                                     const uint8_t* route, uint32_t pack_flags,
+                                     uint32_t* mask_words, uint64_t* counts, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+/* tilemix_attention_fwd over a variable-length batch: every sequence is attended causally on
+ * its own; no score crosses a sequence boundary.  dbg tiles are (sequence, h_q, m, n) with m, n
+ * counted inside the sequence.  Requires every sequence to have at most 2048 key tiles. */
+int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varlen_t* vl,
+                                 const void* q_f16, const void* k_f16, const void* v_f16,
+                                 const int8_t* q_i8, const int8_t* k_i8, const float* q_scale,
+                                 const float* k_scale, const uint32_t* mask_words, void* out_f16,
+                                 float* lse, void* workspace, size_t workspace_bytes,
+                                 const tilemix_debug_t* dbg, void* stream);
+
 /* W = ceil(ceil(L / (G*tile_n)) / 32); <= 0 on invalid arguments. */
 int tilemix_mask_words_per_row(int seqlen, int tile_n, int group);
 /* Bytes of `workspace` needed by tilemix_attention_fwd (0 on an invalid problem). */

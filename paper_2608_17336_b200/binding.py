@@ -21,6 +21,8 @@ EXPORTS = (
     "tilemix_prefill_host",
     "tilemix_mask_words_per_row", "tilemix_workspace_size", "tilemix_scratch_bytes", "tilemix_arena_size",
     "tilemix_read_status", "tilemix_status_string", "tilemix_launch_count",
+    "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
+    "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
 )
 
 
@@ -62,6 +64,11 @@ class DebugStruct(ctypes.Structure):
                 ("kind", ctypes.c_void_p)]
 
 
+class VarlenStruct(ctypes.Structure):
+    _fields_ = [("n_seqs", ctypes.c_int32), ("max_seqlen", ctypes.c_int32),
+                ("cu_seqlens", ctypes.POINTER(ctypes.c_int32))]
+
+
 _lib = None
 
 
@@ -90,6 +97,14 @@ def lib() -> ctypes.CDLL:
         L.tilemix_status_string.argtypes = [i32]
         L.tilemix_status_string.restype = ctypes.c_char_p
         L.tilemix_launch_count.restype = ctypes.c_uint64
+        vlp = ctypes.POINTER(VarlenStruct)
+        L.tilemix_varlen_counts.argtypes = [pp, vlp, ctypes.POINTER(ctypes.c_int64 * 7)]
+        L.tilemix_varlen_workspace_size.argtypes = [pp, vlp]
+        L.tilemix_varlen_workspace_size.restype = ctypes.c_size_t
+        L.tilemix_quantize_qk_varlen.argtypes = [pp, vlp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.tilemix_pack_routing_mask_varlen.argtypes = [pp, vlp, vp, u32, vp, vp, vp, ctypes.c_size_t, vp]
+        L.tilemix_attention_fwd_varlen.argtypes = [pp, vlp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                   ctypes.c_size_t, ctypes.POINTER(DebugStruct), vp]
         _lib = L
     return _lib
 
@@ -226,3 +241,105 @@ def tilemix_workspace_size(p): return int(lib().tilemix_workspace_size(ctypes.by
 def tilemix_scratch_bytes(p): return int(lib().tilemix_scratch_bytes(ctypes.byref(p)))
 def tilemix_mask_words_per_row(seqlen, tile_n, group): return int(lib().tilemix_mask_words_per_row(seqlen, tile_n, group))
 def tilemix_launch_count(): return int(lib().tilemix_launch_count())
+
+
+# ------------------------------------------------------------------ variable-length batches
+
+class Varlen:
+    """Host-side description of a packed batch: keeps the cu_seqlens array alive for the C struct."""
+
+    def __init__(self, cu_seqlens, max_seqlen: int = 0):
+        cu = [int(x) for x in cu_seqlens]
+        self.cu = (ctypes.c_int32 * len(cu))(*cu)
+        self.struct = VarlenStruct(len(cu) - 1, max_seqlen, ctypes.cast(self.cu, ctypes.POINTER(ctypes.c_int32)))
+        self.cu_list = cu
+
+    def ref(self):
+        return ctypes.byref(self.struct)
+
+
+def tilemix_varlen_counts(p: ProblemStruct, vl: Varlen) -> dict:
+    out = (ctypes.c_int64 * 7)()
+    _check(lib().tilemix_varlen_counts(ctypes.byref(p), vl.ref(), ctypes.byref(out)), "tilemix_varlen_counts")
+    keys = ("total", "sum_T_m", "sum_blk_q", "sum_blk_k", "T_mask_max", "W", "max_seqlen")
+    return dict(zip(keys, (int(x) for x in out)))
+
+
+def tilemix_varlen_workspace_size(p: ProblemStruct, vl: Varlen) -> int:
+    return int(lib().tilemix_varlen_workspace_size(ctypes.byref(p), vl.ref()))
+
+
+def _varlen_strides(p: ProblemStruct, q=None, k=None, v=None, o=None) -> ProblemStruct:
+    """Tensors are [total, H, d]; the C struct wants (batch, head, token) strides."""
+    pp = ProblemStruct.from_buffer_copy(p)
+    for name, t in (("q_stride", q), ("k_stride", k), ("v_stride", v), ("o_stride", o)):
+        if t is not None:
+            assert t.dim() == 3 and t.stride(-1) == 1 and t.shape[-1] == p.head_dim
+            f = getattr(pp, name)
+            f[0], f[1], f[2] = 0, t.stride(1), t.stride(0)
+    return pp
+
+
+def _varlen_ws(p, vl, dev, workspace):
+    if workspace is None:
+        workspace = torch.empty(tilemix_varlen_workspace_size(p, vl), dtype=torch.uint8, device=dev)
+    return workspace
+
+
+def tilemix_quantize_qk_varlen(p: ProblemStruct, vl: Varlen, q: torch.Tensor, k: torch.Tensor, workspace=None):
+    """q [total,Hq,d], k [total,Hk,d] FP16 -> (q_i8 [Hq,total,d], k_i8 [Hk,total,d], q_scale [blocks_q,Hq],
+    k_scale [blocks_k,Hk])."""
+    c = tilemix_varlen_counts(p, vl)
+    dev = q.device
+    q8 = torch.empty((p.heads_q, p.seqlen, p.head_dim), dtype=torch.int8, device=dev)
+    k8 = torch.empty((p.heads_kv, p.seqlen, p.head_dim), dtype=torch.int8, device=dev)
+    qs = torch.empty((c["sum_blk_q"], p.heads_q), dtype=torch.float32, device=dev)
+    ks = torch.empty((c["sum_blk_k"], p.heads_kv), dtype=torch.float32, device=dev)
+    ws = _varlen_ws(p, vl, dev, workspace)
+    pp = _varlen_strides(p, q=q, k=k)
+    _check(lib().tilemix_quantize_qk_varlen(ctypes.byref(pp), vl.ref(), _ptr(q), _ptr(k), _ptr(q8), _ptr(k8),
+                                            _ptr(qs), _ptr(ks), _ptr(ws), ws.numel(), _stream()),
+           "tilemix_quantize_qk_varlen")
+    return q8, k8, qs, ks
+
+
+def tilemix_pack_routing_mask_varlen(p: ProblemStruct, vl: Varlen, route: torch.Tensor, pin_diagonal=False,
+                                     workspace=None):
+    """route uint8 [Hk, sum T_m, T_mask_max] -> (words [Hk, sum T_m, W] int32-typed bits, counts int64 [Hk,2])."""
+    c = tilemix_varlen_counts(p, vl)
+    assert route.dtype == torch.uint8 and route.is_cuda and route.is_contiguous()
+    assert tuple(route.shape) == (p.heads_kv, c["sum_T_m"], c["T_mask_max"]), route.shape
+    words = torch.empty((p.heads_kv, c["sum_T_m"], c["W"]), dtype=torch.int32, device=route.device)
+    counts = torch.empty((p.heads_kv, 2), dtype=torch.int64, device=route.device)
+    ws = _varlen_ws(p, vl, route.device, workspace)
+    _check(lib().tilemix_pack_routing_mask_varlen(ctypes.byref(p), vl.ref(), _ptr(route),
+                                                  PIN_DIAGONAL_FP16 if pin_diagonal else 0, _ptr(words),
+                                                  _ptr(counts), _ptr(ws), ws.numel(), _stream()),
+           "tilemix_pack_routing_mask_varlen")
+    return words, counts
+
+
+def tilemix_attention_fwd_varlen(p: ProblemStruct, vl: Varlen, q, k, v, q8=None, k8=None, q_scale=None,
+                                 k_scale=None, words=None, out=None, want_lse=False, debug_tiles=None,
+                                 workspace=None):
+    """Fused forward over a packed batch; q [total,Hq,d], k/v [total,Hk,d].  Returns a dict like
+    tilemix_attention_fwd with out [total,Hq,d] and lse [Hq,total]; debug_tiles are (sequence, h_q, m, n)."""
+    dev = q.device
+    if out is None:
+        out = torch.empty((p.seqlen, p.heads_q, p.head_dim), dtype=torch.float16, device=dev)
+    lse = torch.empty((p.heads_q, p.seqlen), dtype=torch.float32, device=dev) if want_lse else None
+    ws = _varlen_ws(p, vl, dev, workspace)
+    dbg, raw, kind = None, None, None
+    if debug_tiles is not None:
+        tiles = torch.as_tensor(debug_tiles, dtype=torch.int32).reshape(-1, 4).contiguous().to(dev)
+        n = tiles.shape[0]
+        raw = torch.zeros((n, p.tile_m, p.tile_n), dtype=torch.int32, device=dev)
+        kind = torch.full((n,), 255, dtype=torch.uint8, device=dev)
+        dbg = DebugStruct(tiles.data_ptr(), n, raw.data_ptr(), kind.data_ptr())
+    pp = _varlen_strides(p, q=q, k=k, v=v, o=out)
+    rc = lib().tilemix_attention_fwd_varlen(ctypes.byref(pp), vl.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(q8),
+                                            _ptr(k8), _ptr(q_scale), _ptr(k_scale), _ptr(words), _ptr(out),
+                                            _ptr(lse), _ptr(ws), ws.numel(),
+                                            ctypes.byref(dbg) if dbg is not None else None, _stream())
+    _check(rc, "tilemix_attention_fwd_varlen")
+    return {"out": out, "lse": lse, "raw": raw, "kind": kind, "workspace": ws}

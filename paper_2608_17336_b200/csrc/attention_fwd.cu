@@ -86,9 +86,16 @@ struct Params {
     int B, Hq, Hk, L, G, T_m, W, nb;
     int has_int8;                 // INT8 operands present
     float scale_log2;             // softmax scale * log2(e)
-    const float* q_scale;         // [B,Hq,T_m]
-    const float* k_scale;         // [B,Hk,T_n]
+    const float* q_scale;         // [B,Hq,T_m]; variable-length batch: [sum T_m, Hq]
+    const float* k_scale;         // [B,Hk,T_n]; variable-length batch: [sum T_n, Hk]
     const uint32_t* words;        // [nb,Hk,T_m,W] or null (all FP16)
+    // Variable-length batch (null = one dense batch): prefix sums over the sequences.  Then B = 1,
+    // L = total tokens and T_m = total query-tile rows of the packed batch.
+    const int32_t* vl_tok;        // [n_seqs+1] first token of each sequence
+    const int32_t* vl_tile;       // [n_seqs+1] query-tile rows before each sequence
+    const int32_t* vl_item_seq;   // [total_pairs] work item -> sequence (longest rows first)
+    const int32_t* vl_item_pair;  // [total_pairs] work item -> pair of query tiles of that sequence
+    int n_seqs, total_pairs;
     __half* out;
     int64_t os[3];
     float* lse;                   // nullable
@@ -163,7 +170,8 @@ struct Ring {
     __device__ __forceinline__ void flip(uint32_t s) { phases ^= 1u << s; }
 };
 
-template <int D, int T>
+// VL: variable-length batch (the work item is found in the sequence prefix sums).
+template <int D, int T, bool VL>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                  const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16,
@@ -184,13 +192,32 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const long long cta_c0 = clock64();
 #endif
     // ---- work item -------------------------------------------------------------------
-    const int n_pairs = (prm.T_m + 1) >> 1;
-    const int bh = blockIdx.x / n_pairs;
-    const int pr = n_pairs - 1 - (blockIdx.x - bh * n_pairs);   // longest rows first
-    const int b = bh / prm.Hq, hq = bh - b * prm.Hq;
+    // b: batch coordinate of the tensor maps; seq: sequence index (== b for a dense batch);
+    // tok0 / len: first token and length of the sequence; row0: its first row among the mask rows
+    // and scale blocks; m, n below count tiles inside the sequence.
+    int b, hq, pr, seq, tok0 = 0, len = prm.L, row0 = 0, n_rows = prm.T_m;
+    if constexpr (!VL) {
+        const int n_pairs = (prm.T_m + 1) >> 1;
+        const int bh = blockIdx.x / n_pairs;
+        pr = n_pairs - 1 - (blockIdx.x - bh * n_pairs);   // longest rows first
+        b = bh / prm.Hq;
+        hq = bh - b * prm.Hq;
+        seq = b;
+    } else {
+        hq = blockIdx.x / prm.total_pairs;
+        const int item = blockIdx.x - hq * prm.total_pairs;
+        seq = prm.vl_item_seq[item];
+        pr = prm.vl_item_pair[item];
+        b = 0;
+        tok0 = prm.vl_tok[seq];
+        len = prm.vl_tok[seq + 1] - tok0;
+        row0 = prm.vl_tile[seq];
+        n_rows = prm.vl_tile[seq + 1] - row0;
+    }
+    constexpr bool varlen = VL;
     const int hk = hq / (prm.Hq / prm.Hk);
     const int mA = 2 * pr, mB = 2 * pr + 1;
-    const bool hasB = mB < prm.T_m;
+    const bool hasB = mB < n_rows;
     const int nkv = (hasB ? mB : mA) + 1;
 
     // ---- shared memory ------------------------------------------------------------------
@@ -234,7 +261,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if (prm.words != nullptr) {
                 const int g = j / prm.G;
                 const int nbi = (prm.nb == 1) ? 0 : b;
-                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.T_m + mA) * prm.W;
+                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.T_m + row0 + mA) * prm.W;
                 e |= (rowA[g >> 5] >> (g & 31)) & 1u;
                 if (hasB) e |= ((rowA[prm.W + (g >> 5)] >> (g & 31)) & 1u) << 1;
             }
@@ -274,9 +301,9 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 ptx::mbar_arrive_expect_tx(bar_q(t), bytes);
                 for (int c = 0; c < C::kHalves; ++c)
                     ptx::tma_load_4d(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, &tm_q16,
-                                     bar_q(t), c * 64, m * T, hq, b);
+                                     bar_q(t), c * 64, tok0 + m * T, hq, b);
                 if (prm.has_int8)
-                    ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, m * T, hq, b);
+                    ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
             }
             // One ring item = the chunks of one operand tile.  Its data arrives on the "full" barrier
             // of its first chunk; every chunk is handed back on its own "empty" barrier (items of
@@ -287,7 +314,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             bool ok = true;
             auto fill = [&](uint32_t s, int n_chunks, const CUtensorMap* tm, uint32_t bytes, int row) {
                 for (int c = 0; c < n_chunks && ok; ++c) {
-                    if (!wait_bar(cx, bar_empty(s + c), ring.phase(s + c), kRoleProducer, row / T, kBarRingEmpty)) ok = false;
+                    if (!wait_bar(cx, bar_empty(s + c), ring.phase(s + c), kRoleProducer, (row - tok0) / T, kBarRingEmpty)) ok = false;
                     ring.flip(s + c);
                 }
                 if (!ok) return;
@@ -300,9 +327,9 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             };
             for (int j = 0; j < nkv && ok; ++j) {
                 const uint32_t e = sched(j);
-                if (e & 4u) fill(ring.take(C::kHalves), C::kHalves, &tm_k16, C::kHalves * C::kChunk, j * T);
-                if (e & 8u) fill(ring.take(1), 1, &tm_k8, C::kK8Bytes, j * T);
-                fill(ring.take(C::kHalves), C::kHalves, &tm_v16, C::kHalves * C::kChunk, j * T);
+                if (e & 4u) fill(ring.take(C::kHalves), C::kHalves, &tm_k16, C::kHalves * C::kChunk, tok0 + j * T);
+                if (e & 8u) fill(ring.take(1), 1, &tm_k8, C::kK8Bytes, tok0 + j * T);
+                fill(ring.take(C::kHalves), C::kHalves, &tm_v16, C::kHalves * C::kChunk, tok0 + j * T);
             }
             if (!ok || *cx.abort_flag) {
                 // let copies that are still in flight land before the CTA's memory is released
@@ -448,10 +475,17 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
             const uint32_t t_s = lane_base + t * C::kSCols;
             const uint32_t t_o = lane_base + 2 * C::kSCols + t * C::kOCols;
-            const int64_t i_glob = static_cast<int64_t>(m_t) * T + row;
-            const bool row_valid = row < T && i_glob < prm.L;
-            const float dq = prm.has_int8 ? prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t] : 0.f;
-            const float* dk_row = prm.has_int8 ? prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.T_m : nullptr;
+            const int i_loc = m_t * T + row;                         // row inside the sequence
+            const int64_t i_glob = static_cast<int64_t>(tok0) + i_loc;   // row on the token axis
+            const bool row_valid = row < T && i_loc < len;
+            // scales: dense [B,H,T_m] (unit stride over blocks), variable-length [blocks, H]
+            const int64_t dk_step = varlen ? prm.Hk : 1;
+            const float dq = !prm.has_int8 ? 0.f
+                             : varlen ? prm.q_scale[static_cast<int64_t>(row0 + m_t) * prm.Hq + hq]
+                                      : prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t];
+            const float* dk_row = !prm.has_int8 ? nullptr
+                                  : varlen ? prm.k_scale + static_cast<int64_t>(row0) * prm.Hk + hk
+                                           : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.T_m;
             float m_run = -INFINITY, z = 0.f;
             float m_seen = -INFINITY;     // largest scaled score seen so far (m_run may lag it)
             bool ok = true;
@@ -468,7 +502,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     a *= dq * dk_next;
                     if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                 }
-                if (prm.has_int8 && j < m_t) dk_next = dk_row[j + 1];   // next tile's scale, ahead of its use
+                if (prm.has_int8 && j < m_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long sw0 = clock64();
 #endif
@@ -541,7 +575,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         if (lane == 0) {
                             for (int e = 0; e < prm.dbg_n; ++e) {
                                 const int32_t* q = prm.dbg_tiles + 4 * e;
-                                if (q[0] == b && q[1] == hq && q[2] == m_t && q[3] == j) { idx = e; break; }
+                                if (q[0] == seq && q[1] == hq && q[2] == m_t && q[3] == j) { idx = e; break; }
                             }
                         }
                         idx = __shfl_sync(0xffffffffu, idx, 0);
@@ -710,7 +744,8 @@ int encode_map(EncodeTiledFn enc, CUtensorMap* tm, const void* base, int elem_by
 template <int D, int T>
 int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, const int8_t* q8,
                 const int8_t* k8, const float* qs, const float* ks, const uint32_t* words, void* out,
-                float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream) {
+                float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream,
+                const VarlenDev* vl, int total_pairs) {
     using C = Cfg<D, T>;
     EncodeTiledFn enc = nullptr;
     int rc = get_encoder(&enc);
@@ -741,16 +776,23 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     prm.os[0] = g.os[0]; prm.os[1] = g.os[1]; prm.os[2] = g.os[2];
     prm.lse = lse;
     prm.status = static_cast<int*>(workspace);
+    if (vl != nullptr) {
+        prm.vl_tok = vl->tok; prm.vl_tile = vl->tile; prm.vl_item_seq = vl->item_seq; prm.vl_item_pair = vl->item_pair;
+        prm.n_seqs = vl->n; prm.total_pairs = total_pairs;
+    }
     if (dbg != nullptr && dbg->n_tiles > 0) {
         prm.dbg_tiles = dbg->tiles; prm.dbg_n = dbg->n_tiles; prm.dbg_raw = dbg->raw; prm.dbg_kind = dbg->kind;
     }
     cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceClearBytes, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
-    e = cudaFuncSetAttribute(attention_kernel<D, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
+    const auto kernel = vl ? attention_kernel<D, T, true> : attention_kernel<D, T, false>;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
     if (e != cudaSuccess) return static_cast<int>(e);
-    const int64_t ctas = static_cast<int64_t>(g.B) * g.Hq * ((g.T_m + 1) / 2);
+    const int64_t ctas = vl ? static_cast<int64_t>(g.Hq) * total_pairs
+                            : static_cast<int64_t>(g.B) * g.Hq * ((g.T_m + 1) / 2);
+    if (ctas == 0) return TILEMIX_OK;   // only zero-length sequences
     if (ctas > 0x7fffffffLL) return static_cast<int>(cudaErrorInvalidConfiguration);
-    attention_kernel<D, T><<<static_cast<unsigned>(ctas), kThreads, C::kSmemAlloc, stream>>>(prm, tq, tk, tv, tq8, tk8);
+    kernel<<<static_cast<unsigned>(ctas), kThreads, C::kSmemAlloc, stream>>>(prm, tq, tk, tv, tq8, tk8);
     g_launch_count.fetch_add(1);
     return static_cast<int>(cudaGetLastError());
 }
@@ -759,11 +801,14 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
 
 int launch_attention(const Geometry& g, const void* q, const void* k, const void* v, const int8_t* q8,
                      const int8_t* k8, const float* qs, const float* ks, const uint32_t* words, void* out,
-                     float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream) {
+                     float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream,
+                     const VarlenDev* vl, int total_pairs) {
     if (g.d == 128 && g.tile_m == 128)
-        return launch_impl<128, 128>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream);
+        return launch_impl<128, 128>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream, vl,
+                                     total_pairs);
     if (g.d == 64 && g.tile_m == 64)
-        return launch_impl<64, 64>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream);
+        return launch_impl<64, 64>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream, vl,
+                                   total_pairs);
     return TILEMIX_ERR_UNSUPPORTED;
 }
 

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <vector>
 
 #include "tilemix.h"
 
@@ -30,16 +31,58 @@ struct Geometry {
 // Fills `g`; returns TILEMIX_OK or a negative error.  Checks sizes only (no pointers).
 int resolve(const tilemix_problem_t* p, Geometry* g);
 
+// Variable-length batch: host-side prefix sums over the sequences and their device copy.
+struct VarlenTable {
+    int n = 0;                 // sequences
+    int max_len = 0;           // longest sequence (or the caller's bound)
+    int total_tiles = 0, total_pairs = 0, total_blk_q = 0, total_blk_k = 0;
+    // four arrays of n + 1 entries (tok, tile, blkq, blkk), then two of total_pairs entries: the
+    // attention kernel's work items (sequence, pair of query tiles), longest first
+    std::vector<int32_t> tab;
+};
+struct VarlenDev {
+    const int32_t* tok = nullptr;    // first token of sequence s (cu_seqlens)
+    const int32_t* tile = nullptr;   // query-tile rows before sequence s
+    const int32_t* blkq = nullptr;   // quantiser blocks of Q before sequence s
+    const int32_t* blkk = nullptr;   // quantiser blocks of K before sequence s
+    const int32_t* item_seq = nullptr;   // work item -> sequence
+    const int32_t* item_pair = nullptr;  // work item -> pair of query tiles (2p, 2p+1) of that sequence
+    int n = 0;
+};
+constexpr size_t kStatusAreaBytes = 4096;   // status record, timers, trace: start of every workspace
+
+// Fills `g` for the packed batch (B = 1, L = total tokens, T_m = sum of tile rows, T_mask / W of the
+// longest sequence, T_n = key tiles of the longest sequence) and the prefix sums.
+int resolve_varlen(const tilemix_problem_t* p, const tilemix_varlen_t* vl, Geometry* g, VarlenTable* t);
+// Copies the tables behind the status area of `workspace` on `stream` and points `dev` at them.
+int upload_varlen(const VarlenTable& t, void* workspace, cudaStream_t stream, VarlenDev* dev);
+
+#ifdef __CUDACC__
+// Sequence s with off[s] <= x < off[s+1] (off non-decreasing, off[0] <= x < off[n]).
+__device__ __forceinline__ int find_seq(const int32_t* __restrict__ off, int n, int x) {
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+#endif
+
 inline bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 
 // Launchers implemented in the .cu files (all enqueue on `stream`, return cudaError_t as int).
+// `vl` (nullable) switches a launcher to the variable-length layouts; `blk_off` / `total_blk` are the
+// block prefix sums of the operand being quantised.
 int launch_quantize(const void* x, const int64_t stride[3], int B, int H, int L, int d, int blk,
-                    int8_t* out, float* scale, cudaStream_t stream);
+                    int8_t* out, float* scale, cudaStream_t stream, const VarlenDev* vl = nullptr,
+                    const int32_t* blk_off = nullptr, int total_blk = 0);
 int launch_pack(const Geometry& g, const uint8_t* route, uint32_t pack_flags, uint32_t* words,
-                unsigned long long* counts, cudaStream_t stream);
+                unsigned long long* counts, cudaStream_t stream, const VarlenDev* vl = nullptr);
 int launch_attention(const Geometry& g, const void* q, const void* k, const void* v,
                      const int8_t* q8, const int8_t* k8, const float* qs, const float* ks,
                      const uint32_t* words, void* out, float* lse, void* workspace,
-                     const tilemix_debug_t* dbg, cudaStream_t stream);
+                     const tilemix_debug_t* dbg, cudaStream_t stream, const VarlenDev* vl = nullptr,
+                     int total_pairs = 0);
 
 }  // namespace tilemix

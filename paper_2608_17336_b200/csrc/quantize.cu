@@ -49,18 +49,29 @@ __device__ __forceinline__ uint2 quant8(const uint4& v, float delta, float rdelt
     return make_uint2(o[0], o[1]);
 }
 
-// One CTA per (batch*head, block).  MAXV = 16-byte vectors cached per thread; blocks with more
+// One CTA per (batch*head, block).  With a variable-length batch (tok != null) the CTA's block index
+// runs over the blocks of all sequences; the sequence is found in the block prefix sums, blocks
+// restart at each sequence's first token and scales are stored block-major [blocks, H].  MAXV = 16-byte vectors cached per thread; blocks with more
 // than kThreads*MAXV vectors re-read the remainder from global memory (L2) in the second pass.
 template <int MAXV>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, int64_t s_tok,
                 int H, int L, int d, int blk, int n_blk, int8_t* __restrict__ out,
-                float* __restrict__ scale) {
+                float* __restrict__ scale, const int32_t* __restrict__ tok,
+                const int32_t* __restrict__ blk_off, int n_seqs) {
     const int r = blockIdx.x % n_blk;
     const int bh = blockIdx.x / n_blk;
     const int b = bh / H, h = bh % H;
-    const int row0 = r * blk;
-    const int rows = min(blk, L - row0);
+    int row0 = r * blk;
+    int rows = min(blk, L - row0);
+    int64_t scale_idx = static_cast<int64_t>(bh) * n_blk + r;
+    if (tok != nullptr) {
+        const int s = find_seq(blk_off, n_seqs, r);
+        const int r_loc = r - blk_off[s];
+        row0 = tok[s] + r_loc * blk;
+        rows = min(blk, tok[s + 1] - row0);
+        scale_idx = static_cast<int64_t>(r) * H + h;
+    }
     const int vec_per_row = d >> 3;
     const int nvec = rows * vec_per_row;
     const __half* src = x + b * s_batch + h * s_head + static_cast<int64_t>(row0) * s_tok;
@@ -98,7 +109,7 @@ quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, i
     const float amax_f = __half2float(__ushort_as_half(static_cast<unsigned short>(amax)));
     const float delta = __fdiv_rn(amax_f, 127.0f);
     const float rdelta = __frcp_rn(delta);
-    if (threadIdx.x == 0) scale[static_cast<int64_t>(bh) * n_blk + r] = delta;
+    if (threadIdx.x == 0) scale[scale_idx] = delta;
 
     if (amax == 0u) {  // zero block: delta = 0, xhat = 0 (no division by zero)
         for (int v = threadIdx.x; v < nvec; v += kThreads)
@@ -120,8 +131,11 @@ quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, i
 }  // namespace
 
 int launch_quantize(const void* x, const int64_t stride[3], int B, int H, int L, int d, int blk,
-                    int8_t* out, float* scale, cudaStream_t stream) {
-    const int n_blk = static_cast<int>(ceil_div(L, blk));
+                    int8_t* out, float* scale, cudaStream_t stream, const VarlenDev* vl,
+                    const int32_t* blk_off, int total_blk) {
+    const int n_blk = vl ? total_blk : static_cast<int>(ceil_div(L, blk));
+    const int32_t* tok = vl ? vl->tok : nullptr;
+    const int n_seqs = vl ? vl->n : 0;
     const int64_t ctas = static_cast<int64_t>(B) * H * n_blk;
     if (ctas <= 0) return cudaSuccess;
     if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
@@ -130,10 +144,10 @@ int launch_quantize(const void* x, const int64_t stride[3], int B, int H, int L,
     const dim3 grid(static_cast<unsigned>(ctas));
     if (nvec <= kThreads * 2) {
         quantize_kernel<2><<<grid, kThreads, 0, stream>>>(xp, stride[0], stride[1], stride[2], H, L,
-                                                          d, blk, n_blk, out, scale);
+                                                          d, blk, n_blk, out, scale, tok, blk_off, n_seqs);
     } else {
         quantize_kernel<8><<<grid, kThreads, 0, stream>>>(xp, stride[0], stride[1], stride[2], H, L,
-                                                          d, blk, n_blk, out, scale);
+                                                          d, blk, n_blk, out, scale, tok, blk_off, n_seqs);
     }
     g_launch_count.fetch_add(1);
     return static_cast<int>(cudaGetLastError());

@@ -79,3 +79,66 @@ def check_rows(gpu_out: torch.Tensor, ref: np.ndarray, rows, atol=ATOL):
 def all_rows(w: synth.Workload, heads=None):
     heads = range(w.heads) if heads is None else heads
     return [(b, h, i) for b in range(w.batch) for h in heads for i in range(w.seqlen)]
+
+
+# ------------------------------------------------------------------ variable-length batches
+
+def varlen_inputs(cu, heads_q, heads_kv, head_dim, tile, group, seed, int8_fraction=0.5):
+    """Seeded packed batch: q [total,Hq,d], k/v [total,Hk,d] CPU half tensors and a byte map
+    route [Hk, sum T_m, T_mask_max] with Bernoulli(int8_fraction) entries."""
+    total = cu[-1]
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    q = torch.randn((total, heads_q, head_dim), generator=gen).half()
+    k = torch.randn((total, heads_kv, head_dim), generator=gen).half()
+    v = torch.randn((total, heads_kv, head_dim), generator=gen).half()
+    lens = [cu[s + 1] - cu[s] for s in range(len(cu) - 1)]
+    rows = sum(-(-L // tile) for L in lens)
+    t_mask_max = max(1, -(-max(lens) // (group * tile)))
+    rng = np.random.default_rng(seed + 1)
+    route = (rng.random((heads_kv, rows, t_mask_max)) < int8_fraction).astype(np.uint8)
+    return q, k, v, route
+
+
+def varlen_oracle(cu, q, k, v, route, tile, group, pin_diagonal=False, seqs=None):
+    """The dense oracle applied to every sequence of a packed batch on its own (a variable-length
+    batch is, by definition, independent causal problems laid end to end).  Returns one dict per
+    sequence (None for an empty or skipped one) with q8/k8/scales/words/out/lse and its offsets."""
+    Hq, Hk, d = q.shape[1], k.shape[1], q.shape[2]
+    res, row0 = [], 0
+    for s in range(len(cu) - 1):
+        t0, t1 = cu[s], cu[s + 1]
+        L = t1 - t0
+        T_m = -(-L // tile)
+        if L == 0 or (seqs is not None and s not in seqs):
+            res.append(None)
+            row0 += T_m
+            continue
+        p = oracle.Problem(1, Hq, Hk, L, d, tile, tile, group)
+        qb, kb, vb = (np_bits(t[t0:t1].permute(1, 0, 2)[None]) for t in (q, k, v))
+        q8, qs = oracle.quantize(qb, p.bq)
+        k8, ks = oracle.quantize(kb, p.bk)
+        r = np.ascontiguousarray(route[None, :, row0:row0 + T_m, :p.T_mask])
+        words, counts = oracle.pack(p, r, pin_diagonal)
+        out, lse, _ = oracle.attention_full(p, qb, kb, vb, q8, k8, qs, ks, words)
+        res.append(dict(p=p, tok0=t0, row0=row0, q8=q8, k8=k8, qs=qs, ks=ks, words=words, counts=counts,
+                        out=out, lse=lse, qb=qb, kb=kb))
+        row0 += T_m
+    return res
+
+
+def run_gpu_varlen(cu, q, k, v, route, tile, group, pin_diagonal=False, flags=0, debug_tiles=None,
+                   max_seqlen=0):
+    from paper_2608_17336_b200 import binding
+    dev = torch.device("cuda:0")
+    Hq, Hk, d = q.shape[1], k.shape[1], q.shape[2]
+    p = binding.problem(1, Hq, Hk, cu[-1], d, tile, tile, group, flags=flags)
+    vl = binding.Varlen(cu, max_seqlen)
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    q8, k8, qs, ks = binding.tilemix_quantize_qk_varlen(p, vl, qd, kd)
+    words, counts = binding.tilemix_pack_routing_mask_varlen(p, vl, torch.from_numpy(route).to(dev), pin_diagonal)
+    res = binding.tilemix_attention_fwd_varlen(p, vl, qd, kd, vd, q8, k8, qs, ks, words, want_lse=True,
+                                               debug_tiles=debug_tiles)
+    code, rec = binding.tilemix_read_status(res["workspace"])
+    assert code == 0, f"device status {rec}"
+    res.update(q8=q8, k8=k8, qs=qs, ks=ks, words=words, counts=counts, p=p, vl=vl)
+    return res

@@ -110,3 +110,60 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(b, "LIB_PATH", "/nonexistent/libtilemix.so")
     with pytest.raises(RuntimeError, match="no CPU or library fallback"):
         b.lib()
+
+
+# ------------------------------------------------------------------ variable-length batches
+
+def test_varlen_counts_and_workspace(lib):
+    lens = [1, 37, 64, 0, 200, 129, 513]
+    cu = np.cumsum([0] + lens).tolist()
+    p = b.problem(1, 4, 2, cu[-1], 64, 64, 64, group=2)
+    vl = b.Varlen(cu)
+    c = b.tilemix_varlen_counts(p, vl)
+    tiles = sum(-(-L // 64) for L in lens)
+    assert c == dict(total=cu[-1], sum_T_m=tiles, sum_blk_q=tiles, sum_blk_k=tiles,
+                     T_mask_max=-(-513 // 128), W=1, max_seqlen=513)
+    # the paper's scale shapes for variable-length batches: sum_b ceil(L_b / block) entries per head
+    p2 = b.problem(1, 4, 2, cu[-1], 64, 64, 64, quant_blk_q=128, quant_blk_k=32)
+    c2 = b.tilemix_varlen_counts(p2, vl)
+    assert c2["sum_blk_q"] == sum(-(-L // 128) for L in lens)
+    assert c2["sum_blk_k"] == sum(-(-L // 32) for L in lens)
+    # status area + four int32 tables of n_seqs + 1 entries + two int32 per work item (pair of query
+    # tiles: 12 here), rounded up to 256 bytes
+    assert b.tilemix_varlen_workspace_size(p, vl) == 4096 + 256
+    big = b.Varlen(list(range(0, 101)))
+    assert b.tilemix_varlen_workspace_size(b.problem(1, 1, 1, 100, 64, 64, 64), big) == 4096 + 2560   # 4 * 101 * 4 + 2 * 100 * 4 = 2416 bytes
+
+
+def test_varlen_host_side_validation(lib):
+    cu = [0, 100, 300]
+    ok = b.problem(1, 2, 2, 300, 64, 64, 64)
+    out = (ctypes.c_int64 * 7)()
+
+    def counts(p, vl):
+        return lib.tilemix_varlen_counts(ctypes.byref(p), vl.ref() if vl else None, ctypes.byref(out))
+
+    assert counts(ok, b.Varlen(cu)) == b.OK
+    assert counts(ok, None) == b.ERR_NULL
+    assert counts(ok, b.Varlen([0, 100, 299])) == b.ERR_SHAPE          # last entry != seqlen
+    assert counts(ok, b.Varlen([1, 100, 300])) == b.ERR_SHAPE          # first entry != 0
+    assert counts(ok, b.Varlen([0, 200, 100, 300])) == b.ERR_SHAPE     # decreasing
+    assert counts(ok, b.Varlen(cu, max_seqlen=150)) == b.ERR_SHAPE     # bound below the longest sequence
+    assert counts(ok, b.Varlen(cu, max_seqlen=4096)) == b.OK and out[4] == 64 and out[5] == 2
+    assert counts(b.problem(2, 2, 2, 300, 64, 64, 64), b.Varlen(cu)) == b.ERR_SHAPE   # batch must be 1
+    assert lib.tilemix_varlen_workspace_size(ctypes.byref(ok), b.Varlen([0, 1, 2]).ref()) == 0
+    # the launching entry points reject bad arguments before touching the device
+    vl = b.Varlen(cu)
+    one = ctypes.c_void_p(4096)
+    assert lib.tilemix_quantize_qk_varlen(ctypes.byref(ok), vl.ref(), None, None, None, None, None, None,
+                                          one, 8192, None) == b.ERR_NULL
+    assert lib.tilemix_quantize_qk_varlen(ctypes.byref(ok), vl.ref(), one, None, one, None, one, None,
+                                          one, 100, None) == b.ERR_WORKSPACE
+    assert lib.tilemix_pack_routing_mask_varlen(ctypes.byref(ok), vl.ref(), None, 0, one, None, one, 8192,
+                                                None) == b.ERR_NULL
+    assert lib.tilemix_attention_fwd_varlen(ctypes.byref(ok), vl.ref(), one, one, one, None, None, None, None,
+                                            None, one, None, one, 8192, None, None) == b.ERR_NULL
+    long = b.problem(1, 1, 1, 64 * 2049, 64, 64, 64, flags=b.FORCE_FP16)
+    assert lib.tilemix_attention_fwd_varlen(ctypes.byref(long), b.Varlen([0, 64 * 2049]).ref(), one, one, one,
+                                            None, None, None, None, None, one, None, one, 8192, None,
+                                            None) == b.ERR_UNSUPPORTED
