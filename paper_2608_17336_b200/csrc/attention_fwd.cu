@@ -50,7 +50,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kTauSoft = 8.0f, kTauHard = 15.0f, kMargin = 6.0f;
 
 enum Role : int { kRoleSoftmaxA = 0, kRoleSoftmaxB = 1, kRoleProducer = 2, kRoleMma = 3 };
-enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6 };
+enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6, kBarPV = 7 };
 
 template <int D, int T>
 struct Cfg {
@@ -71,7 +71,8 @@ struct Cfg {
     static constexpr int kOffQ8 = 2 * kQ16Tile;
     static constexpr int kOffRing = kOffQ8 + 2 * kQ8Tile;
     static constexpr int kOffBars = kOffRing + kRing * kChunk;
-    static constexpr int kNumBars = 2 + 2 * kRing + 2 + 2 + 2 + 1;
+    static constexpr int kTH = T / 2;                 // key columns per half step
+    static constexpr int kNumBars = 2 + 2 * kRing + 4 + 4 + 2 + 2 + 1;
     static constexpr int kOffMisc = kOffBars + kNumBars * 8;       // tmem base, abort flag
     static constexpr int kOffWords = kOffMisc + 16;
     static constexpr int kSmemBytes = kOffWords + kMaxTiles / 2;   // 4-bit schedule entries
@@ -225,10 +226,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     auto bar_q = [&](int t) { return bar0 + 8u * t; };
     auto bar_full = [&](int s) { return bar0 + 8u * (2 + s); };
     auto bar_empty = [&](int s) { return bar0 + 8u * (2 + kRing + s); };
-    auto bar_s = [&](int t) { return bar0 + 8u * (2 + 2 * kRing + t); };
-    auto bar_p = [&](int t) { return bar0 + 8u * (4 + 2 * kRing + t); };
-    auto bar_o = [&](int t) { return bar0 + 8u * (6 + 2 * kRing + t); };
-    const uint32_t bar_drain = bar0 + 8u * (8 + 2 * kRing);
+    // per query tile t and half h of the score tile: "S half ready", "P half ready"; per tile: "PV retired"
+    auto bar_s = [&](int t, int h) { return bar0 + 8u * (2 + 2 * kRing + 2 * t + h); };
+    auto bar_p = [&](int t, int h) { return bar0 + 8u * (6 + 2 * kRing + 2 * t + h); };
+    auto bar_pv = [&](int t) { return bar0 + 8u * (10 + 2 * kRing + t); };   // every PV of tile t
+    auto bar_o = [&](int t) { return bar0 + 8u * (12 + 2 * kRing + t); };    // the last PV of tile t
+    const uint32_t bar_drain = bar0 + 8u * (14 + 2 * kRing);
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);   // [0] tmem base, [1] abort
     uint32_t* sched_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
     Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status};
@@ -238,14 +241,17 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         ptx::mbar_init(bar_q(1), 1);
         for (int s = 0; s < kRing; ++s) {
             ptx::mbar_init(bar_full(s), 1);
-            ptx::mbar_init(bar_empty(s), 1);
+            ptx::mbar_init(bar_empty(s), hasB ? 2 : 1);   // one arrival per MMA issuer
         }
         for (int t = 0; t < 2; ++t) {
-            ptx::mbar_init(bar_s(t), 1);
-            ptx::mbar_init(bar_p(t), kWarpsPerGroup * 32);
+            for (int h = 0; h < 2; ++h) {
+                ptx::mbar_init(bar_s(t, h), 1);
+                ptx::mbar_init(bar_p(t, h), kWarpsPerGroup * 32);
+            }
+            ptx::mbar_init(bar_pv(t), 1);
             ptx::mbar_init(bar_o(t), 1);
         }
-        ptx::mbar_init(bar_drain, 1);
+        ptx::mbar_init(bar_drain, hasB ? 2 : 1);
         misc[1] = 0;
         ptx::fence_mbar_init();
     }
@@ -282,7 +288,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const uint32_t tmem_base = misc[0];
     auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
-    if (warp >= kMmaWarp + 1) {
+    if (warp >= kMmaWarp + 2 || (warp == kMmaWarp + 1 && !hasB)) {
         ptx::setmaxnreg_dec<kRegsOther>();   // idle warps of the third warpgroup
     } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer
@@ -340,16 +346,24 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ================================================================ MMA issuer
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+        // ================================================================ MMA issuers
+        // One issuing thread per query tile (warp kMmaWarp: tile A, the next warp: tile B).  Both walk
+        // the same sequence of ring items; an item goes back to the producer when both have committed it.
         ptx::setmaxnreg_dec<kRegsOther>();
         if (lane == 0) {
-            constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, C::kM, T);
-            constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, C::kM, T);
+            const int t = warp - kMmaWarp;
+            const int m_t = t ? mB : mA;
+            constexpr int TH = C::kTH;
+            constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, C::kM, TH);
+            constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, C::kM, TH);
             constexpr uint32_t kIdescPV = ptx::instr_desc(1, 0, 0, 1, C::kM, D);
             Ring ring;
             bool ok = true;
-            auto acquire = [&](uint32_t s, int j) {   // wait until chunk s holds its data
+            // Wait until chunk s holds its data.  An issuer waits for EVERY item, also those whose data
+            // it does not read: its arrival on the item's "empty" barrier must not run a ring cycle
+            // ahead of the other issuer's, or two arrivals of one issuer would release the chunk.
+            auto acquire = [&](uint32_t s, int j) {
                 if (!ok) return;
                 if (!wait_bar(cx, bar_full(s), ring.phase(s), kRoleMma, j, kBarRingFull)) ok = false;
                 ring.flip(s);
@@ -362,12 +376,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const uint32_t ring_lo = ptx::desc_lo(sbase + C::kOffRing, 16);
             const uint32_t ring_lo_v = ptx::desc_lo(sbase + C::kOffRing, C::kChunk);
             constexpr uint32_t kChunkLo = C::kChunk >> 4;
-            // S_t = Q_t K_j^T on the route of tile t
-            auto issue_qk = [&](int t, uint32_t int8_route, uint32_t s16, uint32_t s8) {
-                const uint32_t d_tmem = tmem_base + t * C::kSCols;
+            // Half h of S_t = Q_t K_j^T on the route of tile t: keys [h*TH, (h+1)*TH) of the key tile, i.e.
+            // the rows of the K-major operand from byte h*TH*(row pitch) on (a whole number of swizzle atoms).
+            auto issue_qk = [&](int t, int h, uint32_t int8_route, uint32_t s16, uint32_t s8) {
+                const uint32_t d_tmem = tmem_base + t * C::kSCols + h * TH;
                 if (int8_route) {
                     const uint32_t a_lo = ptx::desc_lo(sbase + C::kOffQ8 + t * C::kQ8Tile, 16);
-                    const uint32_t b_lo = ring_lo + s8 * kChunkLo;
+                    const uint32_t b_lo = ring_lo + s8 * kChunkLo + ((h * TH * C::kI8RowBytes) >> 4);
                     ptx::mma_i8_ss<false>(d_tmem, a_lo, kHi8, b_lo, kHi8, kIdescQK8);
 #pragma unroll
                     for (int k = 1; k < D / 32; ++k)
@@ -376,7 +391,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 #pragma unroll
                     for (int c = 0; c < C::kHalves; ++c) {
                         const uint32_t a_lo = ptx::desc_lo(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, 16);
-                        const uint32_t b_lo = ring_lo + (s16 + c) * kChunkLo;
+                        const uint32_t b_lo = ring_lo + (s16 + c) * kChunkLo + ((h * TH * 128) >> 4);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             if (c == 0 && k == 0)
@@ -387,38 +402,40 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     }
                 }
             };
-            // O_t (+)= P_t V_j with P in tensor memory (two FP16 per 32-bit column)
-            auto issue_pv = [&](int t, uint32_t sv, uint32_t accumulate) {
+            // O_t (+)= P_t V_j over the keys of half h, with P in tensor memory (two FP16 per 32-bit
+            // column, at the start of its own half of S_t)
+            auto issue_pv = [&](int t, int h, uint32_t sv, uint32_t accumulate) {
                 const uint32_t d_tmem = tmem_base + 2 * C::kSCols + t * C::kOCols;
-                const uint32_t a_tmem = tmem_base + t * C::kSCols;
-                const uint32_t b_lo = ring_lo_v + sv * kChunkLo;
+                const uint32_t a_tmem = tmem_base + t * C::kSCols + h * TH;
+                const uint32_t b_lo = ring_lo_v + sv * kChunkLo + h * (TH / 16) * 128;
                 ptx::mma_f16_ts(d_tmem, a_tmem, b_lo, kHi16, kIdescPV, accumulate);
 #pragma unroll
-                for (int k = 1; k < T / 16; ++k)
+                for (int k = 1; k < TH / 16; ++k)
                     ptx::mma_f16_ts(d_tmem, a_tmem + k * 8, b_lo + k * 128, kHi16, kIdescPV, 1u);
             };
 
-            for (int t = 0; t < (hasB ? 2 : 1) && ok; ++t)
-                if (!wait_bar(cx, bar_q(t), 0, kRoleMma, t, kBarQ)) ok = false;
+            if (!wait_bar(cx, bar_q(t), 0, kRoleMma, t, kBarQ)) ok = false;
 
             // slots of the K operands of the tile whose QK^T is issued next
             uint32_t e_next = sched(0), k16 = 0, k8 = 0;
+            uint32_t r_next = (e_next >> t) & 1u;          // route of this tile at the next key tile
             if (e_next & 4u) { k16 = ring.take(C::kHalves); acquire(k16, 0); }
             if (e_next & 8u) { k8 = ring.take(1); acquire(k8, 0); }
             if (ok) {
                 ptx::tc_fence_after_sync();
-                issue_qk(0, e_next & 1u, k16, k8);
-                ptx::mma_commit(bar_s(0));
-                if (hasB) {
-                    issue_qk(1, e_next & 2u, k16, k8);
-                    ptx::mma_commit(bar_s(1));
+                for (int h = 0; h < 2; ++h) {
+                    issue_qk(t, h, r_next, k16, k8);
+                    ptx::mma_commit(bar_s(t, h));
                 }
                 if (e_next & 4u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
                 if (e_next & 8u) ptx::mma_commit(bar_empty(k8));
             }
             for (int j = 0; j < nkv && ok; ++j) {
+                const bool mine = j <= m_t;            // tile A has no work at the last key tile of tile B
+                const bool more = j + 1 <= m_t;
                 const uint32_t sv = ring.take(C::kHalves);
                 e_next = (j + 1 < nkv) ? sched(j + 1) : 0u;
+                r_next = (e_next >> t) & 1u;
                 if (e_next & 4u) k16 = ring.take(C::kHalves);
                 if (e_next & 8u) k8 = ring.take(1);
                 // operands of this iteration: wait for them now, off the P -> PV critical path
@@ -426,34 +443,30 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (e_next & 4u) acquire(k16, j + 1);
                 if (e_next & 8u) acquire(k8, j + 1);
                 if (!ok) break;
+                // Half steps: as soon as P of a half has arrived its PV is issued, and right behind it the
+                // QK^T of the NEXT key tile into the same half of S_t -- the softmax group is meanwhile
+                // working on the other half.
+                if (mine) {
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    const int m_t = t ? mB : mA;
-                    if ((t == 1 && !hasB) || j > m_t) continue;
-#ifdef TILEMIX_PHASE_TIMERS
-                    const long long mw0 = clock64();
+                    for (int h = 0; h < 2; ++h) {
+#if defined(TILEMIX_TRACE) && !defined(TILEMIX_TRACE4)
+                        if (blockIdx.x == 5 && j >= 8 && j < 8 + 16)
+                            reinterpret_cast<long long*>(cx.status)[320 + ((j - 8) * 4 + 2 * h + t) * 2 + 1] = clock64();
 #endif
-                    if (!wait_bar(cx, bar_p(t), j & 1, kRoleMma, j, kBarP)) { ok = false; break; }
-#ifdef TILEMIX_PHASE_TIMERS
-                    const long long mw1 = clock64();
-                    TM_TIMER_ADD(45, mw1 - mw0);
+                        if (!wait_bar(cx, bar_p(t, h), j & 1, kRoleMma, j, kBarP)) { ok = false; break; }
+#if defined(TILEMIX_TRACE) && !defined(TILEMIX_TRACE4)
+                        if (blockIdx.x == 5 && j >= 8 && j < 8 + 16)
+                            reinterpret_cast<long long*>(cx.status)[320 + ((j - 8) * 4 + 2 * h + t) * 2] = clock64();
 #endif
-                    ptx::tc_fence_after_sync();
-                    issue_pv(t, sv, j > 0);
-                    if (j == m_t) ptx::mma_commit(bar_o(t));
-#ifdef TILEMIX_PHASE_TIMERS
-                    const long long mw3 = clock64();
-#endif
-                    if (j + 1 <= m_t) {
-                        issue_qk(t, e_next & (1u << t), k16, k8);
-                        ptx::mma_commit(bar_s(t));
+                        ptx::tc_fence_after_sync();
+                        issue_pv(t, h, sv, (j > 0 || h > 0) ? 1u : 0u);
+                        ptx::mma_commit(bar_pv(t));
+                        if (j == m_t && h == 1) ptx::mma_commit(bar_o(t));
+                        if (more) {
+                            issue_qk(t, h, r_next, k16, k8);
+                            ptx::mma_commit(bar_s(t, h));
+                        }
                     }
-#ifdef TILEMIX_PHASE_TIMERS
-                    const long long mw5 = clock64();
-                    TM_TIMER_ADD(46, mw5 - mw1);
-                    TM_TIMER_ADD(47, 1);
-                    TM_TIMER_ADD(49, mw3 - mw1); TM_TIMER_ADD(51, mw5 - mw3);
-#endif
                 }
                 if (!ok) break;
                 for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(sv + c));
@@ -495,47 +508,64 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const long long loop_c0 = clock64();
 #endif
             float dk_next = prm.has_int8 ? dk_row[0] : 0.f;
-            for (int j = 0; j <= m_t; ++j) {
-                const uint32_t int8_route = (sched(j) >> t) & 1u;
-                float a = prm.scale_log2;
-                if (int8_route) {
-                    a *= dq * dk_next;
-                    if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
+            float a = prm.scale_log2;
+            uint32_t int8_route = 0u;
+            constexpr int TH = C::kTH;
+            const int n_steps = 2 * (m_t + 1);
+            // One step = one half (TH key columns) of a score tile: while this group works on one half
+            // of S_t, the tensor pipe runs the PV of the previous half and the QK^T of the next one
+            // into the other half.  u = 2*j + h.
+            // While a one-pass step is still computing, the first 32 columns of the next step are put in
+            // flight if that S half is already there (it normally is): `prefetched`.
+            uint32_t first[32];
+            bool prefetched = false;
+            for (int u = 0; u < n_steps; ++u) {
+                const int j = u >> 1, h = u & 1;
+                if (h == 0) {
+                    int8_route = (sched(j) >> t) & 1u;
+                    a = prm.scale_log2;
+                    if (int8_route) {
+                        a *= dq * dk_next;
+                        if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
+                    }
+                    if (prm.has_int8 && j < m_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
                 }
-                if (prm.has_int8 && j < m_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
+                const uint32_t t_sh = t_s + h * TH;
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long sw0 = clock64();
 #endif
-                ok = wait_bar(cx, bar_s(t), j & 1, role, j, kBarS);
+                if (!prefetched) {
+                    ok = wait_bar(cx, bar_s(t, h), j & 1, role, j, kBarS);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                }
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(39, clock64() - sw0);
 #endif
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st0 = clock64();
 #endif
 #ifdef TILEMIX_TRACE
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && j >= 8 && j < 8 + 48)
-                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2] = clock64();
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
+                    reinterpret_cast<long long*>(cx.status)[128 + ((u - 16) * 2 + t) * 2] = clock64();
 #endif
 
                 // ---- shared online-softmax state (Sec. 3.1), log2 domain --------------------------
-                // P = 2^(a*raw - m) is rounded to FP16 and packed two per word into p2[0 .. T/2).
-                // The running maximum m is lazy: it moves only when a tile exceeds it by more than
-                // kTau.  So an interior tile is done in ONE pass with the current m, 32 columns at a
+                // P = 2^(a*raw - m) is rounded to FP16 and packed two per word into p2[0 .. TH/2).
+                // The running maximum m is lazy: it moves only when a step exceeds it by more than
+                // kTau.  So an interior step is done in ONE pass with the current m, 32 columns at a
                 // time with the next 32 already in flight from tensor memory, while its row maximum is
                 // tracked on the side; only if some row of the warp does exceed m + kTau (rare after
-                // the first tiles) the tile is re-read and redone in the generic two-pass form.
+                // the first tiles) the half tile is re-read and redone in the generic two-pass form.
                 const bool diag = (j == m_t);
                 bool redo = diag || j == 0 || prm.dbg_n > 0;
                 float alpha = 1.f, sum = 0.f;
                 bool grow = false;
-                uint32_t p2[T / 2];
+                uint32_t p2[TH / 2];
                 if (__any_sync(0xffffffffu, m_seen > m_run + kTauSoft)) {
-                    // Deferred move of the maximum decided on the previous tile (all rows of the warp):
-                    // z changes scale here, O~ below together with any move this tile itself forces.
+                    // Deferred move of the maximum decided on an earlier step (all rows of the warp):
+                    // z changes scale here, O~ below together with any move this step itself forces.
 #ifdef TILEMIX_TRACE
                     if (lane == 0) atomicAdd(&cx.status[21], 1);
 #endif
@@ -550,8 +580,20 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 #endif
                 if (!redo) {
                     float mx;
-                    if (int8_route) softmax_tile_fast<T, true>(t_s, a, m_run, p2, sum, mx);
-                    else softmax_tile_fast<T, false>(t_s, a, m_run, p2, sum, mx);
+                    if (!prefetched) ptx::tmem_ld32(t_sh, first);
+                    prefetched = false;
+                    // next step: one-pass as well (not the first or the diagonal tile), and its S half ready?
+                    const int jn = (u + 1) >> 1, hn = (u + 1) & 1;
+                    const bool next_fast = u + 1 < n_steps && jn != m_t;
+                    auto late = [&]() {
+                        if (next_fast && __all_sync(0xffffffffu, ptx::mbar_test_wait(bar_s(t, hn), jn & 1))) {
+                            ptx::tc_fence_after_sync();
+                            ptx::tmem_ld32(t_s + hn * TH, first);
+                            prefetched = true;
+                        }
+                    };
+                    if (int8_route) softmax_tile_fast<TH, true>(t_sh, first, a, m_run, p2, sum, mx, late);
+                    else softmax_tile_fast<TH, false>(t_sh, first, a, m_run, p2, sum, mx, late);
                     const float m_tile = mx * a;
                     redo = __any_sync(0xffffffffu, m_tile > m_run + kTauHard);   // P would overflow FP16
                     if (!redo) m_seen = fmaxf(m_seen, m_tile);
@@ -559,16 +601,19 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st2 = clock64() + (__float_as_int(sum) & 0);
 #endif
-#ifdef TILEMIX_TRACE
+#ifdef TILEMIX_TRACE4
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
+                    reinterpret_cast<long long*>(cx.status)[320 + ((u - 16) * 2 + t) * 2] = clock64() + (__float_as_int(sum) & 0);
+#elif defined(TILEMIX_TRACE)
                 if (lane == 0) { atomicAdd(&cx.status[22], 1); if (redo) atomicAdd(&cx.status[20], 1); }
 #endif
                 if (redo) {
-                    // Generic two-pass form: first and diagonal tiles, tiles that move the maximum, and
-                    // every tile in debug mode.  The raw accumulators are (still) in tensor memory.
-                    uint32_t s[T];
+                    // Generic two-pass form: first and diagonal tiles, steps that move the maximum, and
+                    // every step in debug mode.  The raw accumulators are (still) in tensor memory.
+                    uint32_t s[TH];
 #pragma unroll
-                    for (int c = 0; c < T / 32; ++c)
-                        ptx::tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+                    for (int c = 0; c < TH / 32; ++c)
+                        ptx::tmem_ld32(t_sh + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
                     ptx::tmem_wait_ld();
                     if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
                         int idx = -1;
@@ -580,9 +625,9 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         }
                         idx = __shfl_sync(0xffffffffu, idx, 0);
                         if (idx >= 0 && row < T) {
-                            int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + row) * T;
+                            int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + row) * T + h * TH;
 #pragma unroll
-                            for (int c = 0; c < T; c += 4)
+                            for (int c = 0; c < TH; c += 4)
                                 *reinterpret_cast<uint4*>(dst + c) = make_uint4(s[c], s[c + 1], s[c + 2], s[c + 3]);
                             if (row == 0) prm.dbg_kind[idx] = static_cast<uint8_t>(int8_route);
                         }
@@ -591,14 +636,14 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     // enforced kernel-side, independent of R), row maximum, then the exponentials.
                     float mx = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < T; ++c) {
+                    for (int c = 0; c < TH; ++c) {
                         float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
-                        if (diag && c > row) v = -INFINITY;
+                        if (diag && h * TH + c > row) v = -INFINITY;
                         s[c] = __float_as_uint(v);
                         mx = fmaxf(mx, v);
                     }
                     const float m_tile = mx * a;     // a >= 0, so max(a*raw) = a*max(raw)
-                    // generic form: move at once (to the largest score seen, this tile included)
+                    // generic form: move at once (to the largest score seen, this step included)
                     m_seen = fmaxf(m_seen, m_tile);
                     float a_now = 1.f;
                     if (m_seen > m_run + kTauSoft) {
@@ -609,7 +654,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
                     float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int c = 0; c < T; c += 2) {
+                    for (int c = 0; c < TH; c += 2) {
                         const float2 t2 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), a2, nm2);
                         const float2 pp = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
                         acc = __fadd2_rn(acc, pp);
@@ -624,9 +669,15 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 const long long st3 = clock64() + (__float_as_int(z) & 0);
 #endif
 
-                if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                    // O~ *= alpha.  PV of tile j-1 has retired: it was issued before the QK^T
-                    // whose completion this group has just observed.
+                if (u > 0 && __any_sync(0xffffffffu, grow)) {
+                    // O~ *= alpha.  The PV of the previous step may still be accumulating into O~: wait
+                    // until it has retired (the PV of this step is not issued before P arrives below).
+                    // The S half seen above was issued behind PV(u-2), so that barrier is in phase u-1
+                    // or u and its parity is unambiguous.
+                    ok = wait_bar(cx, bar_pv(t), (u - 1) & 1, role, j, kBarPV);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[32];
@@ -637,15 +688,21 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         ptx::tmem_st32(t_o + c * 32, o);
                     }
                 }
-#pragma unroll
-                for (int c = 0; c < T / 64; ++c)
-                    ptx::tmem_st32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&p2[c * 32]));
+                if constexpr (TH / 2 == 32) {
+                    ptx::tmem_st32(t_sh, p2);
+                } else {
+                    ptx::tmem_st16(t_sh, p2);
+                }
                 ptx::tmem_wait_st();
+#ifdef TILEMIX_TRACE4
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
+                    reinterpret_cast<long long*>(cx.status)[320 + ((u - 16) * 2 + t) * 2 + 1] = clock64();
+#endif
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(bar_p(t));
+                ptx::mbar_arrive(bar_p(t, h));
 #ifdef TILEMIX_TRACE
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && j >= 8 && j < 8 + 48)
-                    reinterpret_cast<long long*>(cx.status)[128 + ((j - 8) * 2 + t) * 2 + 1] = clock64();
+                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
+                    reinterpret_cast<long long*>(cx.status)[128 + ((u - 16) * 2 + t) * 2 + 1] = clock64();
 #endif
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) {

@@ -54,16 +54,19 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     return r;
 }
 
-// One interior score tile in one pass: raw accumulators in tensor memory at t_s -> P = 2^(a*raw - m)
-// rounded to FP16 and packed two per word into p2, the FP32 row sum of P and the row maximum of the
-// raw values.  The 32-column chunks are double-buffered (the next one is in flight while this one is
-// processed), and the per-pair work is software-pipelined in program order -- exponentials of pair
-// k, conversion of pair k + kD1, sum and packing of pair k - (kD2 - kD1) -- because a warp issues in
-// order: the special-function unit takes 16 clocks per pair and the other ~7 instructions of a pair
-// fit in its shadow only if they belong to other pairs.
-template <int T, bool INT8>
-__device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, float a, float m_run, uint32_t (&p2)[T / 2],
-                                                  float& sum, float& mx) {
+// One interior step (T score columns) in one pass: raw accumulators in tensor memory at t_s ->
+// P = 2^(a*raw - m) rounded to FP16 and packed two per word into p2, the FP32 row sum of P and the row
+// maximum of the raw values.  The 32-column chunks are double-buffered (the next one is in flight
+// while this one is processed; the FIRST one was put in flight into `first` by the caller), and the
+// per-pair work is software-pipelined in program order -- exponentials of pair k, conversion of pair
+// k + kD1, sum and packing of pair k - (kD2 - kD1) -- because a warp issues in order: the
+// special-function unit takes 16 clocks per pair and the other ~7 instructions of a pair fit in its
+// shadow only if they belong to other pairs.  `late()` is called once, when `first` is free again (its
+// last chunk has been consumed): the caller may start the NEXT step's first chunk into it there, so
+// that the latency of that load hides behind the rest of this step.
+template <int T, bool INT8, class Late>
+__device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, uint32_t (&first)[32], float a, float m_run,
+                                                  uint32_t (&p2)[T / 2], float& sum, float& mx, Late&& late) {
     // Pipeline depth in pairs: pair k is read (and, INT8, re-biased) in iteration k, made a float in
     // k + 1, scaled in k + 2, exponentiated in k + kE and summed / packed in k + kS.  No instruction
     // uses a result produced in its own iteration.
@@ -74,10 +77,16 @@ __device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, float a, float m
     int mi[4] = {INT_MIN, INT_MIN, INT_MIN, INT_MIN};
     float mf[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     float2 xb[4], tb[4], eb[8];       // rings: biased / float raw values, scaled values, exponentials
-    uint32_t buf[2][32];
-    ptx::tmem_ld32(t_s, buf[0]);
+#ifndef TILEMIX_LATE_BEFORE_END
+#define TILEMIX_LATE_BEFORE_END 8
+#endif
+    // iteration at which late() runs: not before the last even chunk (held in `first`) is consumed
+    constexpr int kFirstFree = ((((T / 32) - 1) & ~1) + 1) * 16;
+    constexpr int kLateAt = (NP - TILEMIX_LATE_BEFORE_END > kFirstFree) ? NP - TILEMIX_LATE_BEFORE_END : kFirstFree;
+    uint32_t buf[32];                 // odd chunks; even chunks land in `first`
 #pragma unroll
     for (int i = 0; i < NP + kS; ++i) {
+        if (i == kLateAt) late();
         if (i >= kE && i - kE < NP) {                         // exponentials of pair i - kE
             const int k = i - kE;
             if (kPolyEvery > 0 && (k % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1)
@@ -96,10 +105,15 @@ __device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, float a, float m
         if (i < NP) {                                         // read pair i
             const int c = i / 16, e = (i % 16) * 2;
             if (e == 0) {
-                ptx::tmem_wait_ld_dep(buf[c & 1]);
-                if (c + 1 < T / 32) ptx::tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1) & 1]);
+                if (c & 1) {
+                    ptx::tmem_wait_ld_dep(buf);
+                    if (c + 1 < T / 32) ptx::tmem_ld32(t_s + (c + 1) * 32, first);
+                } else {
+                    ptx::tmem_wait_ld_dep(first);
+                    if (c + 1 < T / 32) ptx::tmem_ld32(t_s + (c + 1) * 32, buf);
+                }
             }
-            const uint32_t r0 = buf[c & 1][e], r1 = buf[c & 1][e + 1];
+            const uint32_t r0 = (c & 1) ? buf[e] : first[e], r1 = (c & 1) ? buf[e + 1] : first[e + 1];
             if (INT8) {
                 // int -> float without the conversion unit: bits(1.5*2^23) + i is the float
                 // 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D); subtracting 1.5*2^23 is exact.
