@@ -70,7 +70,11 @@ __device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, uint32_t (&first
     // Pipeline depth in pairs: pair k is read (and, INT8, re-biased) in iteration k, made a float in
     // k + 1, scaled in k + 2, exponentiated in k + kE and summed / packed in k + kS.  No instruction
     // uses a result produced in its own iteration.
-    constexpr int NP = T / 2, kE = 3, kS = 7;
+    #ifndef TILEMIX_KE
+#define TILEMIX_KE 3
+#define TILEMIX_KS 7
+#endif
+    constexpr int NP = T / 2, kE = TILEMIX_KE, kS = TILEMIX_KS;
     const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
     const float2 unbias = make_float2(-12582912.f, -12582912.f);
     float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
