@@ -219,6 +219,50 @@ def varlen_leg(tm, w: synth.Workload, dev, peaks) -> dict:
             "unit": "TFLOP/s"}
 
 
+def decode_leg(tm, w: synth.Workload, dev, peaks) -> dict:
+    """One decode step over an INT8 key/value cache of the workload's length: 8 sequences, the workload's
+    heads as query heads over a quarter as many KV heads (GQA 4:1), Bernoulli routing at the workload's
+    INT8 fraction.  HBM-bound: reported against the measured copy bandwidth.  Not part of `value`."""
+    B, Hq, Hk, d, L = 8, w.heads, max(1, w.heads // 4), w.head_dim, w.seqlen
+    gen = torch.Generator(device=dev).manual_seed(w.seed + 11)
+    k = torch.randn((B, Hk, L, d), generator=gen, device=dev, dtype=torch.float16)
+    v = torch.randn((B, Hk, L, d), generator=gen, device=dev, dtype=torch.float16)
+    q = torch.randn((B, Hq, d), generator=gen, device=dev, dtype=torch.float16)
+    k8, v8, ks, vs = tm.tilemix_quantize_qk(tm.problem(B, Hk, Hk, L, d, w.tile, w.tile), k, v)
+    del v
+    T_mask = -(-L // (w.tile * w.group))
+    rng = np.random.default_rng(w.seed + 12)
+    route = (rng.random((1, Hk, T_mask)) < w.int8_fraction)
+    words = np.zeros((1, Hk, -(-T_mask // 32)), np.uint32)
+    for g in range(T_mask):
+        words[..., g >> 5] |= route[..., g].astype(np.uint32) << np.uint32(g & 31)
+    f8 = float(route.mean())
+    words_d = torch.from_numpy(words.view(np.int32)).to(dev)
+    lens = torch.full((B,), L, dtype=torch.int32, device=dev)
+    p = tm.decode_problem(B, Hq, Hk, d, L, w.tile, w.group)
+    work = torch.empty(tm.tilemix_decode_workspace_size(p), dtype=torch.uint8, device=dev)
+    out = torch.empty((B, Hq, d), dtype=torch.float16, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words_d, lens, out=out, workspace=work)
+    n = 10
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for _ in range(n):
+        tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words_d, lens, out=out, workspace=work)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / n
+    # algorithmic bytes: per cached token d (V8) + d (K8, INT8 route) or 2d (FP16 K, FP16 route)
+    nbytes = float(B) * Hk * L * d * (1.0 + f8 + 2.0 * (1.0 - f8))
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"batch": B, "heads_q": Hq, "heads_kv": Hk, "cache_len": L, "int8_groups": f8, "ms_per_step": ms,
+            "tokens_per_s": B / (ms * 1e-3), "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
+            "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "bytes_per_step": nbytes,
+            "l2": "cache (0.8 GB) exceeds L2"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -234,6 +278,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the INT8-fraction sweep of the attention kernel")
     ap.add_argument("--no-varlen", action="store_true", help="skip the variable-length (packed batch) measurement")
+    ap.add_argument("--no-decode", action="store_true", help="skip the INT8 KV-cache decode measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tilemix" else args.warmup
 
@@ -414,6 +459,8 @@ def main():
         line["int8_sweep"] = sweep
     if world == 1 and not args.no_varlen and w.tile == 128:
         line["varlen"] = varlen_leg(tm, w, dev, peaks)
+    if world == 1 and not args.no_decode and w.tile == 128:
+        line["decode"] = decode_leg(tm, w, dev, peaks)
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
         line["cpu_baseline"] = {"value": 4.0 * w.head_dim * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": threads,

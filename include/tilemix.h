@@ -218,6 +218,51 @@ int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varle
                                  float* lse, void* workspace, size_t workspace_bytes,
                                  const tilemix_debug_t* dbg, void* stream);
 
+/* ---- decode step over an INT8 key/value cache (App. C, "Additional Execution Interfaces") ------
+ * One new query token per sequence attends to the first cache_len[b] keys of a cache that holds,
+ * per KV head, K in FP16 and in INT8 and V in INT8, with one FP32 scale per block of tile_n tokens
+ * (the blockwise quantiser above; V is quantised like K, e.g. by passing it to
+ * tilemix_quantize_qk as the K operand).  Bit g of the mask row of (nb, h_k) routes the keys
+ * [g*G*tile_n, (g+1)*G*tile_n):
+ *   bit 1:  s_j = delta_q delta_K[blk(j)] (q8 . k8_j) * scale   -- INT8 dot products, INT32 sums;
+ *           q8, delta_q = the blockwise quantiser applied to the query row, done in the kernel
+ *   bit 0:  s_j = (q . k16_j) * scale                           -- FP16 inputs, FP32 sums
+ * and  o = sum_j softmax(s)_j * delta_V[blk(j)] * v8_j : V8 is converted on chip and its block
+ * scale is folded into the probability before the PV sum (FP32 accumulation), O is written as FP16.
+ * Only the K copy a group is routed to is read, so the bytes per cached token are 2*d (INT8 route)
+ * or 3*d (FP16 route).  The keys are split over n_splits CTAs per (b, h_k); every CTA serves the
+ * H_q/H_k query heads of its KV head; a second kernel merges the partial results.
+ * Supported: head_dim 64 or 128, tile_n 64 or 128, H_q/H_k in {1, 2, 4, 8}. */
+typedef struct tilemix_decode {
+    int32_t batch, heads_q, heads_kv, head_dim;
+    int32_t max_len;       /* token capacity of the caches (their token stride)             */
+    int32_t tile_n, group; /* key tile = scale block; G key tiles per routing bit           */
+    int32_t mask_batch;    /* 1 = one mask row per KV head shared by the batch, or == batch */
+    int32_t n_splits;      /* CTAs per (b, h_k); 0 = chosen by the library                  */
+    float softmax_scale;   /* <= 0 means 1/sqrt(head_dim)                                   */
+} tilemix_decode_t;
+
+/* Bytes of `workspace` for tilemix_decode_int8kv: the partial results of the splits
+ * (0 on an invalid problem). */
+size_t tilemix_decode_workspace_size(const tilemix_decode_t* p);
+/*   q_f16      FP16 [B, Hq, d]
+ *   k_f16      FP16 [B, Hk, max_len, d]   (may be NULL if every legal group is INT8-routed:
+ *                                          a 0 bit then reads NULL -- the caller's contract)
+ *   k_i8, v_i8 INT8 [B, Hk, max_len, d];  k_scale, v_scale FP32 [B, Hk, ceil(max_len/tile_n)]
+ *   mask_words uint32 [nb, Hk, W], W = ceil(ceil(max_len/(G*tile_n))/32); NULL = all FP16
+ *   cache_len  int32 [B] on the DEVICE, 0 <= cache_len[b] <= max_len; a sequence of length 0
+ *              gets an all-zero output row and lse = -inf
+ *   out_f16    FP16 [B, Hq, d];  lse nullable FP32 [B, Hq]
+ *   q_i8_out / q_scale_out  nullable INT8 [B, Hq, d] / FP32 [B, Hq]: the quantised query the
+ *              kernel used (for checking)
+ * Two kernels are enqueued on `stream`.  Errors as for the other entry points. */
+int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const void* k_f16,
+                          const int8_t* k_i8, const float* k_scale, const int8_t* v_i8,
+                          const float* v_scale, const uint32_t* mask_words,
+                          const int32_t* cache_len, void* out_f16, float* lse, int8_t* q_i8_out,
+                          float* q_scale_out, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
 /* W = ceil(ceil(L / (G*tile_n)) / 32); <= 0 on invalid arguments. */
 int tilemix_mask_words_per_row(int seqlen, int tile_n, int group);
 /* Bytes of `workspace` needed by tilemix_attention_fwd (0 on an invalid problem). */

@@ -23,6 +23,7 @@ EXPORTS = (
     "tilemix_read_status", "tilemix_status_string", "tilemix_launch_count",
     "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
     "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
+    "tilemix_decode_workspace_size", "tilemix_decode_int8kv",
 )
 
 
@@ -69,6 +70,11 @@ class VarlenStruct(ctypes.Structure):
                 ("cu_seqlens", ctypes.POINTER(ctypes.c_int32))]
 
 
+class DecodeStruct(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("batch", "heads_q", "heads_kv", "head_dim", "max_len", "tile_n",
+                                               "group", "mask_batch", "n_splits")] + [("softmax_scale", ctypes.c_float)]
+
+
 _lib = None
 
 
@@ -97,6 +103,10 @@ def lib() -> ctypes.CDLL:
         L.tilemix_status_string.argtypes = [i32]
         L.tilemix_status_string.restype = ctypes.c_char_p
         L.tilemix_launch_count.restype = ctypes.c_uint64
+        dp = ctypes.POINTER(DecodeStruct)
+        L.tilemix_decode_workspace_size.argtypes = [dp]
+        L.tilemix_decode_workspace_size.restype = ctypes.c_size_t
+        L.tilemix_decode_int8kv.argtypes = [dp] + [vp] * 12 + [vp, ctypes.c_size_t, vp]
         vlp = ctypes.POINTER(VarlenStruct)
         L.tilemix_varlen_counts.argtypes = [pp, vlp, ctypes.POINTER(ctypes.c_int64 * 7)]
         L.tilemix_varlen_workspace_size.argtypes = [pp, vlp]
@@ -343,3 +353,36 @@ def tilemix_attention_fwd_varlen(p: ProblemStruct, vl: Varlen, q, k, v, q8=None,
                                             ctypes.byref(dbg) if dbg is not None else None, _stream())
     _check(rc, "tilemix_attention_fwd_varlen")
     return {"out": out, "lse": lse, "raw": raw, "kind": kind, "workspace": ws}
+
+
+# ------------------------------------------------------------------ decode over an INT8 KV cache
+
+def decode_problem(batch, heads_q, heads_kv, head_dim, max_len, tile_n, group=1, mask_batch=1, n_splits=0,
+                   softmax_scale=0.0) -> DecodeStruct:
+    return DecodeStruct(batch, heads_q, heads_kv, head_dim, max_len, tile_n, group, mask_batch, n_splits,
+                        softmax_scale)
+
+
+def tilemix_decode_workspace_size(p: DecodeStruct) -> int:
+    return int(lib().tilemix_decode_workspace_size(ctypes.byref(p)))
+
+
+def tilemix_decode_int8kv(p: DecodeStruct, q, k16, k8, k_scale, v8, v_scale, words, cache_len, out=None,
+                          want_lse=False, want_q8=False, workspace=None):
+    """One decode step: q [B,Hq,d] FP16; k16 [B,Hk,max_len,d] FP16 or None; k8/v8 INT8 like k16;
+    scales FP32 [B,Hk,blocks]; words int32-typed bits [nb,Hk,W] or None; cache_len int32 [B] (CUDA).
+    Returns a dict: out [B,Hq,d] FP16, lse, q8, q_scale (if asked)."""
+    dev = q.device
+    if out is None:
+        out = torch.empty((p.batch, p.heads_q, p.head_dim), dtype=torch.float16, device=dev)
+    lse = torch.empty((p.batch, p.heads_q), dtype=torch.float32, device=dev) if want_lse else None
+    q8 = torch.empty((p.batch, p.heads_q, p.head_dim), dtype=torch.int8, device=dev) if want_q8 else None
+    qs = torch.empty((p.batch, p.heads_q), dtype=torch.float32, device=dev) if want_q8 else None
+    if workspace is None:
+        workspace = torch.empty(tilemix_decode_workspace_size(p), dtype=torch.uint8, device=dev)
+    assert cache_len.dtype == torch.int32 and cache_len.is_cuda
+    rc = lib().tilemix_decode_int8kv(ctypes.byref(p), _ptr(q), _ptr(k16), _ptr(k8), _ptr(k_scale), _ptr(v8),
+                                     _ptr(v_scale), _ptr(words), _ptr(cache_len), _ptr(out), _ptr(lse), _ptr(q8),
+                                     _ptr(qs), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "tilemix_decode_int8kv")
+    return {"out": out, "lse": lse, "q8": q8, "q_scale": qs, "workspace": workspace}

@@ -82,6 +82,15 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 
+// Untiled bulk copy global -> shared memory (no multicast): both addresses 16-byte aligned, `bytes` a
+// multiple of 16; completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
 // ---------------------------------------------------------------- register reallocation
 // Executed by every warp of a warpgroup (4 consecutive warps): hands registers back / takes more.
 template <int N>

@@ -167,3 +167,30 @@ def test_varlen_host_side_validation(lib):
     assert lib.tilemix_attention_fwd_varlen(ctypes.byref(long), b.Varlen([0, 64 * 2049]).ref(), one, one, one,
                                             None, None, None, None, None, one, None, one, 8192, None,
                                             None) == b.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ decode over an INT8 KV cache
+
+def test_decode_host_side_validation(lib):
+    ok = b.decode_problem(8, 32, 8, 128, 32768, 128, 4)
+    size = lib.tilemix_decode_workspace_size(ctypes.byref(ok))
+    # 256-byte status area + partial outputs and two float arrays per (batch, query head, split)
+    splits = (size - 256) // (8 * 32 * (128 * 4 + 8))
+    assert splits >= 1 and size == 256 + 8 * 32 * splits * (128 * 4 + 8)
+    assert b.tilemix_decode_workspace_size(b.decode_problem(1, 4, 1, 64, 64, 64, n_splits=7)) == 256 + 1024 + 2 * 256
+    for bad in (b.decode_problem(0, 32, 8, 128, 1024, 128), b.decode_problem(1, 6, 4, 128, 1024, 128),
+                b.decode_problem(1, 4, 4, 128, 0, 128), b.decode_problem(2, 4, 4, 128, 1024, 128, mask_batch=3)):
+        assert lib.tilemix_decode_workspace_size(ctypes.byref(bad)) == 0
+    one = ctypes.c_void_p(4096)
+
+    def call(p, q=one, k16=one, k8=one, ks=one, v8=one, vs=one, words=one, lens=one, out=one, ws=one, nbytes=1 << 30):
+        return lib.tilemix_decode_int8kv(ctypes.byref(p), q, k16, k8, ks, v8, vs, words, lens, out, None, None, None,
+                                         ws, nbytes, None)
+
+    assert call(b.decode_problem(1, 4, 4, 96, 1024, 128)) == b.ERR_UNSUPPORTED      # head_dim
+    assert call(b.decode_problem(1, 12, 4, 128, 1024, 128)) == b.ERR_UNSUPPORTED    # 3 query heads per KV head
+    assert call(b.decode_problem(1, 4, 4, 128, 1024, 32)) == b.ERR_UNSUPPORTED      # tile
+    assert call(ok, q=None) == b.ERR_NULL and call(ok, lens=None) == b.ERR_NULL
+    assert call(ok, k16=None, words=None) == b.ERR_NULL                               # all FP16 without an FP16 cache
+    assert call(ok, k8=ctypes.c_void_p(4100)) == b.ERR_ALIGN
+    assert call(ok, nbytes=size - 1) == b.ERR_WORKSPACE

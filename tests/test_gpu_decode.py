@@ -1,0 +1,100 @@
+"""Decode step over an INT8 key/value cache on the GPU against the float64 oracle: the quantised
+query bit-exact, outputs and LSE within tolerance."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import decode as od
+from tests.helpers import ATOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(B, Hq, Hk, L, d, tile, G, seed, lens, f8=0.5, mask_batch=1):
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    q = torch.randn((B, Hq, d), generator=gen).half()
+    k = torch.randn((B, Hk, L, d), generator=gen).half()
+    v = torch.randn((B, Hk, L, d), generator=gen).half()
+    rng = np.random.default_rng(seed + 1)
+    T_mask = -(-L // (tile * G))
+    route = (rng.random((mask_batch, Hk, T_mask)) < f8).astype(np.uint8)
+    return q, k, v, route, np.asarray(lens, np.int32)
+
+
+def _gpu(q, k, v, route, lens, tile, G, n_splits=0, k16_none=False):
+    from paper_2608_17336_b200 import binding as tm
+    dev = torch.device("cuda:0")
+    B, Hq, d = q.shape
+    Hk, L = k.shape[1], k.shape[2]
+    # the cache is quantised with the library's own blockwise quantiser (K and V as its two operands)
+    pq = tm.problem(B, Hk, Hk, L, d, tile, tile)
+    kd, vd = k.to(dev), v.to(dev)
+    k8, v8, ks, vs = tm.tilemix_quantize_qk(pq, kd, vd)
+    p = tm.decode_problem(B, Hq, Hk, d, L, tile, G, mask_batch=route.shape[0], n_splits=n_splits)
+    words = torch.from_numpy(od.pack_row(route).view(np.int32)).to(dev)
+    res = tm.tilemix_decode_int8kv(p, q.to(dev), None if k16_none else kd, k8, ks, v8, vs, words,
+                                   torch.from_numpy(lens).to(dev), want_lse=True, want_q8=True)
+    torch.cuda.synchronize()
+    return res, dict(k8=k8.cpu().numpy(), ks=ks.cpu().numpy(), v8=v8.cpu().numpy(), vs=vs.cpu().numpy())
+
+
+def _check(q, k, v, route, lens, tile, G, **kw):
+    res, cache = _gpu(q, k, v, route, lens, tile, G, **kw)
+    q16 = np.ascontiguousarray(q.view(torch.int16).numpy()).view(np.uint16)
+    k16 = np.ascontiguousarray(k.view(torch.int16).numpy()).view(np.uint16)
+    # the cache itself: the library quantiser against the oracle's (bit-exact)
+    k8_ref, ks_ref = oracle.quantize(k16, tile)
+    assert np.array_equal(cache["k8"], k8_ref) and np.array_equal(cache["ks"].view(np.uint32), ks_ref.view(np.uint32))
+    q8_ref, dq_ref = od.quantize_query(q16)
+    assert np.array_equal(res["q8"].cpu().numpy(), q8_ref)
+    assert np.array_equal(res["q_scale"].cpu().numpy().view(np.uint32), dq_ref.view(np.uint32))
+    ref, ref_lse = od.decode(q16, k16, cache["k8"], cache["ks"], cache["v8"], cache["vs"], od.pack_row(route), lens,
+                             tile, G)
+    out = res["out"].float().cpu().numpy().astype(np.float64)
+    err = np.abs(out - ref)
+    assert (err <= ATOL * np.maximum(1.0, np.abs(ref))).all(), f"max err {err.max():.3e}"
+    lse = res["lse"].cpu().numpy().astype(np.float64)
+    live = lens > 0
+    assert np.abs(lse[live] - ref_lse[live]).max() < 2e-3
+    assert np.isneginf(lse[~live]).all() and not out[~live].any()
+    return float(err.max())
+
+
+def test_decode_gqa4_d128():
+    q, k, v, route, lens = _case(3, 8, 2, 1500, 128, 128, 2, seed=21, lens=[1500, 777, 129])
+    _check(q, k, v, route, lens, 128, 2)
+
+
+def test_decode_small_tiles_mha_edge_lengths():
+    q, k, v, route, lens = _case(5, 2, 2, 300, 64, 64, 1, seed=22, lens=[300, 1, 0, 64, 65])
+    _check(q, k, v, route, lens, 64, 1)
+
+
+@pytest.mark.parametrize("rep", [1, 2, 8])
+def test_decode_group_sizes(rep):
+    q, k, v, route, lens = _case(2, 2 * rep, 2, 900, 128, 64, 3, seed=23 + rep, lens=[900, 450])
+    _check(q, k, v, route, lens, 64, 3)
+
+
+@pytest.mark.parametrize("n_splits", [1, 3, 1000])
+def test_decode_split_counts(n_splits):
+    q, k, v, route, lens = _case(1, 4, 1, 2000, 64, 128, 1, seed=24, lens=[1999])
+    _check(q, k, v, route, lens, 128, 1, n_splits=n_splits)
+
+
+def test_decode_per_batch_mask_and_pure_routes():
+    q, k, v, route, lens = _case(2, 4, 2, 700, 128, 128, 1, seed=25, lens=[700, 300], mask_batch=2)
+    _check(q, k, v, route, lens, 128, 1)
+    _check(q, k, v, np.zeros_like(route), lens, 128, 1)
+    _check(q, k, v, np.ones_like(route), lens, 128, 1, k16_none=True)    # all INT8: no FP16 cache needed
+
+
+def test_decode_keys_beyond_cache_len_are_not_read():
+    q, k, v, route, lens = _case(1, 4, 1, 512, 128, 128, 1, seed=26, lens=[200])
+    a, _ = _gpu(q, k, v, route, lens, 128, 1)
+    k2, v2 = k.clone(), v.clone()
+    k2[:, :, 256:] = 5.0       # later blocks only: the scales of the blocks in use are unchanged
+    v2[:, :, 256:] = -7.0
+    b_, _ = _gpu(q, k2, v2, route, lens, 128, 1)
+    assert torch.equal(a["out"].view(torch.int16), b_["out"].view(torch.int16))
