@@ -147,8 +147,12 @@ int tilemix_attention_fwd_noalloc(const tilemix_problem_t* p, const void* q_f16,
                                   const tilemix_debug_t* dbg, void** workspace_out, void* stream);
 
 /* Whole path on HOST buffers: copies Q, K, V and the routing map to the device arena,
- * quantises, packs, runs the fused kernel and copies O back; everything is enqueued on
- * `stream` in order (use pinned host memory for the copies to be asynchronous).
+ * quantises, packs, runs the fused kernel and copies O back (use pinned host memory for the
+ * copies to be asynchronous).  The batch -- for a single sequence, its KV heads -- is cut into up
+ * to 8 chunks that are pipelined: host->device copies and device->host copies run on two helper
+ * streams of the library (created on the first call on a device, kept until exit) while the
+ * kernels run on `stream`.  All of it is ordered after the work `stream` held on entry, and
+ * `stream` is made to wait for the last copy, so synchronising `stream` completes the call.
  *   q_host,k_host,v_host  host FP16, dense [B,H,L,d];  route_host host uint8 [nb,Hk,T_m,T_mask]
  *   out_host              host FP16, dense [B,Hq,L,d]
  *   arena                 device scratch of >= tilemix_arena_size(p) bytes, 256-byte aligned */

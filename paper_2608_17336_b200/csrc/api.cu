@@ -185,6 +185,42 @@ size_t tilemix_arena_size(const tilemix_problem_t* p) {
     return arena_layout(g).total;
 }
 
+namespace {
+
+// Helper streams and events of tilemix_prefill_host, created on first use per device and kept until
+// the process exits (stream/event creation is not a device-memory allocation and does not synchronise).
+constexpr int kMaxChunks = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, landed[kMaxChunks] = {}, done[kMaxChunks] = {}, drained = nullptr;
+};
+HostPipe g_pipe[64];
+std::atomic<int> g_pipe_lock{0};
+
+int host_pipe(HostPipe** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    if (dev < 0 || dev >= 64) return TILEMIX_ERR_UNSUPPORTED;
+    HostPipe& hp = g_pipe[dev];
+    while (g_pipe_lock.exchange(1, std::memory_order_acquire) != 0) {}
+    int rc = TILEMIX_OK;
+    if (!hp.ready) {
+        auto ev = [&](cudaEvent_t* x) { if (rc == 0) rc = static_cast<int>(cudaEventCreateWithFlags(x, cudaEventDisableTiming)); };
+        if (rc == 0) rc = static_cast<int>(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+        if (rc == 0) rc = static_cast<int>(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+        ev(&hp.start); ev(&hp.drained);
+        for (int i = 0; i < kMaxChunks; ++i) { ev(&hp.landed[i]); ev(&hp.done[i]); }
+        hp.ready = rc == 0;
+    }
+    g_pipe_lock.store(0, std::memory_order_release);
+    *out = &hp;
+    return rc;
+}
+
+}  // namespace
+
 int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const void* k_host, const void* v_host,
                          const uint8_t* route_host, uint32_t pack_flags, void* out_host, void* arena,
                          size_t arena_bytes, void* stream) {
@@ -199,28 +235,82 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
     if (arena_bytes < a.total) return TILEMIX_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* base = static_cast<uint8_t*>(arena);
-    const size_t nq = static_cast<size_t>(g.B) * g.Hq * g.L * g.d, nk = static_cast<size_t>(g.B) * g.Hk * g.L * g.d;
+    HostPipe* hp = nullptr;
+    if ((rc = host_pipe(&hp))) return rc;
+
+    // The batch (or, for one sequence, its KV heads) is cut into chunks that flow through three
+    // engines at once: host->device copies on a helper stream, the three kernels on the caller's
+    // stream, device->host copies on a second helper stream.  Everything is ordered behind what the
+    // caller's stream held on entry, and the caller's stream ends up behind the last copy.
+    const bool by_batch = g.B > 1;
+    const int units = by_batch ? g.B : g.Hk;
+    const int per_chunk = static_cast<int>(ceil_div(units, kMaxChunks));
+    const int n_chunks = static_cast<int>(ceil_div(units, per_chunk));
+    const int rep = g.Hq / g.Hk;
+    const size_t head_elems = static_cast<size_t>(g.L) * g.d;
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(base + a.q, q_host, nq * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
-    if ((e = cudaMemcpyAsync(base + a.k, k_host, nk * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
-    if ((e = cudaMemcpyAsync(base + a.v, v_host, nk * 2, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+    if ((e = cudaEventRecord(hp->start, s)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess) return e;
+    // routing map: small, copied and packed once for the whole problem
     if ((e = cudaMemcpyAsync(base + a.route, route_host, static_cast<size_t>(g.nb) * g.Hk * g.T_m * g.T_mask,
                              cudaMemcpyHostToDevice, s)) != cudaSuccess)
         return e;
-    tilemix_problem_t dense = *p;
-    if ((rc = tilemix_quantize_qk(&dense, base + a.q, base + a.k, reinterpret_cast<int8_t*>(base + a.q8),
-                                  reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
-                                  reinterpret_cast<float*>(base + a.ks), stream)))
-        return rc;
-    if ((rc = tilemix_pack_routing_mask(&dense, base + a.route, pack_flags, reinterpret_cast<uint32_t*>(base + a.words),
+    if ((rc = tilemix_pack_routing_mask(p, base + a.route, pack_flags, reinterpret_cast<uint32_t*>(base + a.words),
                                         nullptr, stream)))
         return rc;
-    if ((rc = tilemix_attention_fwd(&dense, base + a.q, base + a.k, base + a.v, reinterpret_cast<int8_t*>(base + a.q8),
-                                    reinterpret_cast<int8_t*>(base + a.k8), reinterpret_cast<float*>(base + a.qs),
-                                    reinterpret_cast<float*>(base + a.ks), reinterpret_cast<uint32_t*>(base + a.words),
-                                    base + a.o, nullptr, base + a.work, 4096, nullptr, stream)))
-        return rc;
-    if ((e = cudaMemcpyAsync(out_host, base + a.o, nq * 2, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return e;
+    for (int c = 0; c < n_chunks; ++c) {
+        const int u0 = c * per_chunk, nu = (u0 + per_chunk <= units ? per_chunk : units - u0);
+        // element offsets of the chunk inside the dense [B, H, L, d] tensors, and its byte counts
+        const size_t q_off = by_batch ? static_cast<size_t>(u0) * g.Hq * head_elems : static_cast<size_t>(u0) * rep * head_elems;
+        const size_t k_off = by_batch ? static_cast<size_t>(u0) * g.Hk * head_elems : static_cast<size_t>(u0) * head_elems;
+        const size_t q_n = by_batch ? static_cast<size_t>(nu) * g.Hq * head_elems : static_cast<size_t>(nu) * rep * head_elems;
+        const size_t k_n = by_batch ? static_cast<size_t>(nu) * g.Hk * head_elems : static_cast<size_t>(nu) * head_elems;
+        const uint8_t* qh = static_cast<const uint8_t*>(q_host) + q_off * 2;
+        const uint8_t* kh = static_cast<const uint8_t*>(k_host) + k_off * 2;
+        const uint8_t* vh = static_cast<const uint8_t*>(v_host) + k_off * 2;
+        if ((e = cudaMemcpyAsync(base + a.q + q_off * 2, qh, q_n * 2, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return e;
+        if ((e = cudaMemcpyAsync(base + a.k + k_off * 2, kh, k_n * 2, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return e;
+        if ((e = cudaMemcpyAsync(base + a.v + k_off * 2, vh, k_n * 2, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess) return e;
+        if ((e = cudaEventRecord(hp->landed[c], hp->in)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(s, hp->landed[c], 0)) != cudaSuccess) return e;
+        // the chunk as a problem of its own: a batch range (dense) or a head range (strides of the whole)
+        tilemix_problem_t sub = *p;
+        size_t words_off = 0, qs_off = 0, ks_off = 0;
+        if (by_batch) {
+            sub.batch = nu;
+            sub.mask_batch = g.nb == 1 ? 1 : nu;
+            words_off = g.nb == 1 ? 0 : static_cast<size_t>(u0) * g.Hk * g.T_m * g.W;
+            qs_off = static_cast<size_t>(u0) * g.Hq * ceil_div(g.L, g.blk_q);
+            ks_off = static_cast<size_t>(u0) * g.Hk * ceil_div(g.L, g.blk_k);
+        } else {
+            sub.heads_kv = nu;
+            sub.heads_q = nu * rep;
+            for (int t = 0; t < 3; ++t) {
+                sub.q_stride[t] = g.qs[t]; sub.k_stride[t] = g.ks[t]; sub.v_stride[t] = g.vs[t]; sub.o_stride[t] = g.os[t];
+            }
+            words_off = static_cast<size_t>(u0) * g.T_m * g.W;
+            qs_off = static_cast<size_t>(u0) * rep * ceil_div(g.L, g.blk_q);
+            ks_off = static_cast<size_t>(u0) * ceil_div(g.L, g.blk_k);
+        }
+        int8_t* q8 = reinterpret_cast<int8_t*>(base + a.q8) + q_off;
+        int8_t* k8 = reinterpret_cast<int8_t*>(base + a.k8) + k_off;
+        float* qs = reinterpret_cast<float*>(base + a.qs) + qs_off;
+        float* ks = reinterpret_cast<float*>(base + a.ks) + ks_off;
+        if ((rc = tilemix_quantize_qk(&sub, base + a.q + q_off * 2, base + a.k + k_off * 2, q8, k8, qs, ks, stream)))
+            return rc;
+        if ((rc = tilemix_attention_fwd(&sub, base + a.q + q_off * 2, base + a.k + k_off * 2, base + a.v + k_off * 2, q8, k8,
+                                        qs, ks, reinterpret_cast<uint32_t*>(base + a.words) + words_off,
+                                        base + a.o + q_off * 2, nullptr, base + a.work, 4096, nullptr, stream)))
+            return rc;
+        if ((e = cudaEventRecord(hp->done[c], s)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(hp->out, hp->done[c], 0)) != cudaSuccess) return e;
+        if ((e = cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + q_off * 2, base + a.o + q_off * 2, q_n * 2,
+                                 cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
+            return e;
+    }
+    if ((e = cudaEventRecord(hp->drained, hp->out)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(s, hp->drained, 0)) != cudaSuccess) return e;
     return TILEMIX_OK;
 }
 

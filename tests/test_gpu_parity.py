@@ -314,3 +314,31 @@ def test_full_size_config_sampled_rows(name, override, n_heads, n_tiles, n_rows)
     assert torch.isfinite(out).all()
     vmax = v.abs().amax(dim=(2, 3)).cuda()
     assert (out.abs().amax(dim=(2, 3)) <= vmax * (1 + 1e-2)).all()
+
+
+@pytest.mark.parametrize("B,Hq,Hk,nb", [(1, 12, 6, 1), (1, 20, 10, 1), (3, 4, 2, 1), (11, 2, 2, 11)])
+def test_prefill_host_equals_device_path(B, Hq, Hk, nb):
+    """The host-buffer entry point (chunks pipelined over helper streams) returns, bit for bit, what
+    the three device calls return; more than eight chunk units, GQA, shared and per-batch masks."""
+    from paper_2608_17336_b200 import binding
+    L, d, tile, G = 300, 64, 64, 2
+    gen = torch.Generator(device="cpu").manual_seed(77 + B)
+    q = torch.randn((B, Hq, L, d), generator=gen).half()
+    k = torch.randn((B, Hk, L, d), generator=gen).half()
+    v = torch.randn((B, Hk, L, d), generator=gen).half()
+    p = binding.problem(B, Hq, Hk, L, d, tile, tile, G, mask_batch=nb)
+    rng = np.random.default_rng(5)
+    route = (rng.random((nb, Hk, p.T_m, p.T_mask)) < 0.5).astype(np.uint8)
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    q8, k8, qs, ks = binding.tilemix_quantize_qk(p, qd, kd)
+    words, _ = binding.tilemix_pack_routing_mask(p, torch.from_numpy(route).to(dev), True)
+    ref = binding.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words)["out"].cpu()
+    arena = torch.empty(binding.tilemix_arena_size(p), dtype=torch.uint8, device=dev)
+    out = torch.empty((B, Hq, L, d), dtype=torch.float16).pin_memory()
+    for _ in range(2):     # a second call right behind the first reuses the helper streams and the arena
+        out.zero_()
+        binding.tilemix_prefill_host(p, q.pin_memory(), k.pin_memory(), v.pin_memory(),
+                                     torch.from_numpy(route).pin_memory(), out, arena, pin_diagonal=True)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
