@@ -93,16 +93,21 @@ quantize_kernel(const __half* __restrict__ x, int64_t s_batch, int64_t s_head, i
     const __half* src = x + b * s_batch + h * s_head + static_cast<int64_t>(row0) * s_tok;
     int8_t* dst = out + (static_cast<int64_t>(bh) * L + row0) * d;
 
+    // (row, 16-byte chunk) of this thread's i-th vector, v = threadIdx.x + i * kThreads, kept
+    // incrementally: one division per thread instead of one per vector
+    const int step_row = kThreads / vec_per_row, step_c8 = kThreads % vec_per_row;
+    const int row_first = threadIdx.x / vec_per_row, c8_first = threadIdx.x - row_first * vec_per_row;
     uint4 cache[MAXV > 0 ? MAXV : 1];
     uint32_t amax2 = 0u;
+    int row = row_first, c8 = c8_first;
 #pragma unroll
     for (int i = 0; i < MAXV; ++i) {
         const int v = threadIdx.x + i * kThreads;
         cache[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (v < nvec) {
-            const int row = v / vec_per_row, c8 = v - row * vec_per_row;
-            cache[i] = __ldg(reinterpret_cast<const uint4*>(src + row * s_tok + c8 * 8));
-        }
+        if (v < nvec) cache[i] = __ldg(reinterpret_cast<const uint4*>(src + row * s_tok + c8 * 8));
+        row += step_row;
+        c8 += step_c8;
+        if (c8 >= vec_per_row) { c8 -= vec_per_row; ++row; }
         amax2 = umax2(amax2, umax2(umax2(habs2_bits(cache[i].x), habs2_bits(cache[i].y)),
                                    umax2(habs2_bits(cache[i].z), habs2_bits(cache[i].w))));
     }
