@@ -204,15 +204,19 @@ decode_kernel(const DecodeParams prm) {
             if (int8) {
                 uint4 kq = make_uint4(0u, 0u, 0u, 0u);
                 if (j < len) kq = *reinterpret_cast<const uint4*>(kst + key * D + 16 * c);
+                int dot[R];
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    int dot = __dp4a(static_cast<int>(kq.x), static_cast<int>(q8r[r].x), 0);
-                    dot = __dp4a(static_cast<int>(kq.y), static_cast<int>(q8r[r].y), dot);
-                    dot = __dp4a(static_cast<int>(kq.z), static_cast<int>(q8r[r].z), dot);
-                    dot = __dp4a(static_cast<int>(kq.w), static_cast<int>(q8r[r].w), dot);
+                    dot[r] = __dp4a(static_cast<int>(kq.x), static_cast<int>(q8r[r].x), 0);
+                    dot[r] = __dp4a(static_cast<int>(kq.y), static_cast<int>(q8r[r].y), dot[r]);
+                    dot[r] = __dp4a(static_cast<int>(kq.z), static_cast<int>(q8r[r].z), dot[r]);
+                    dot[r] = __dp4a(static_cast<int>(kq.w), static_cast<int>(q8r[r].w), dot[r]);
+                }
 #pragma unroll
-                    for (int o = CH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    s[r] = static_cast<float>(dot) * (prm.scale_log2 * dq_s[r] * dkt);
+                for (int r = 0; r < R; ++r) {
+#pragma unroll
+                    for (int o = CH / 2; o > 0; o >>= 1) dot[r] += __shfl_xor_sync(0xffffffffu, dot[r], o);
+                    s[r] = static_cast<float>(dot[r]) * (prm.scale_log2 * dq_s[r] * dkt);
                 }
             } else {
                 uint4 k0 = make_uint4(0u, 0u, 0u, 0u), k1 = k0;
@@ -420,9 +424,10 @@ int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     g->W = static_cast<int>(ceil_div(g->T_mask, 32));
     int splits = p->n_splits;
     if (splits == 0) {
-        // two waves of two CTAs per SM over the whole batch (measured: more splits cost more in
-        // per-CTA set-up and merge than they gain in tail), at least two key tiles per split
-        const int64_t want = ceil_div(148 * 2 * 2, static_cast<int64_t>(p->batch) * p->heads_kv);
+        // at most two full waves of two CTAs per SM over the whole batch (measured: more splits cost
+        // more in per-CTA set-up and merge than they gain, and a third, partial wave idles a quarter
+        // of the GPU), at least two key tiles per split
+        const int64_t want = (148 * 2 * 2) / (static_cast<int64_t>(p->batch) * p->heads_kv);
         splits = static_cast<int>(want < 1 ? 1 : want);
         const int cap = g->n_blk / 2 > 0 ? g->n_blk / 2 : 1;
         if (splits > cap) splits = cap;
