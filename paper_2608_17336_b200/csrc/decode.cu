@@ -21,6 +21,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 struct DecodeParams {
     int B, Hq, Hk, max_len, G, nb, W, n_splits, n_blk;
+    int tile_n;      // tokens per scale block and per routing key tile (a multiple of the kernel's chunk)
     float scale_log2;
     const __half* q;
     const __half* k16;
@@ -51,7 +52,7 @@ __device__ __forceinline__ void bytes_to_floats(uint32_t w, float2 (&f)[2]) {
                                   __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653))), bias);
 }
 
-constexpr int kStages = 2;                 // ring of key/value tiles in shared memory
+constexpr int kStages = 2;                 // ring of key/value chunks in shared memory
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 
 template <int D, int T>
@@ -72,24 +73,49 @@ __device__ __forceinline__ bool wait_tile(uint32_t bar, uint32_t parity) {
     return true;
 }
 
-// D: head dim; R: query heads per KV head; T: key tile (= scale block).
-// Key/value tiles are contiguous in the cache, so one thread streams them into a ring of shared-
-// memory stages with untiled bulk copies a tile ahead of their use; with two CTAs per SM this keeps
-// ~64 KB per SM in flight.  Per tile: (1) scores of all 256 threads from the K stage, (2) the online
-// softmax of each query row by one warp, (3) the PV sums from the V stage.
+// ---- warp-level tensor-core MMAs (m16n8k32 INT8 / m16n8k16 FP16, FP32 or INT32 accumulators) ----------
+// Lane l holds, with g = l / 4 and t = l % 4: A rows g (a0, a2) and g + 8 (a1, a3), B column g, C rows g
+// (c0, c1) and g + 8 (c2, c3) at columns 2t, 2t + 1.  Only rows 0..R-1 of A are query rows here, so a1 and
+// a3 are always zero and c2, c3 stay zero.
+__device__ __forceinline__ void mma_s8(int (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// D: head dim; R: query heads per KV head; T: keys per chunk (the scale block / routing tile tile_n is a
+// multiple of it).  Chunks are contiguous in the cache, so one thread streams them into a ring of
+// shared-memory stages with untiled bulk copies, kStages - 1 chunks ahead of their use; with two CTAs
+// per SM this keeps 100-150 KB per SM in flight.  Per chunk:
+//  (1) scores S[R x T] = Q K^T on the tensor cores, the R query rows being rows 0..R-1 of a 16-row A
+//      operand; each warp takes T/8 keys.  The contraction index may be permuted freely as long as Q and K
+//      use the same permutation, so lane t simply takes the 16-byte chunks t, t+4, ... of a row.
+//  (2) the online softmax of each query row by one warp; P gets delta_V and is rounded to FP16.
+//  (3) O~[R x D] += P V8 on the tensor cores; each warp takes 16 keys (T = 128) and all columns.  V8 is
+//      converted to FP16 in registers (exactly); the output columns are permuted (column n of block nb
+//      is d = (D/8) n + nb) so that the bytes a lane needs from a cached row are contiguous.
 template <int D, int R, int T>
-__global__ void __launch_bounds__(kThreads, (R <= 4 ? 2 : 1))
+__global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(const DecodeParams prm) {
-    constexpr int CH = D / 16;           // 16-byte chunks (lanes) per cached row
-    constexpr int KPP = kThreads / CH;   // keys per pass of the CTA
-    constexpr int KPT = T / KPP;         // keys per thread per tile
     using St = Stage<D, T>;
-    static_assert(KPT >= 1 && T % KPP == 0, "tile too small for the thread mapping");
-    static_assert(kStages * St::kBytes >= static_cast<int>(kThreads / 32 * R * D * sizeof(float)),
+    constexpr int kWarps = kThreads / 32;
+    constexpr int NB1 = T / 8 / kWarps;           // key blocks (8 keys) per warp in phase 1
+    constexpr int W8 = D / 16, W16 = D / 8;       // 32-bit words per lane and row: INT8 / FP16 operand
+    constexpr int KS3 = T / 16;                   // 16-key steps of a tile in phase 3
+    constexpr int NSPLIT = kWarps / KS3;          // warps sharing one such step (each takes some column blocks)
+    constexpr int NBLK = D / 8 / NSPLIT;          // column blocks per warp in phase 3
+    constexpr int BPG = D / 8;                    // bytes of a cached V row per lane group
+    static_assert(NB1 >= 1 && KS3 <= kWarps && kWarps % KS3 == 0, "tile shape vs warps");
+    static_assert(kStages * St::kBytes >= static_cast<int>(kWarps * R * D * sizeof(float)),
                   "the final reduction reuses the ring");
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slot = tid / CH, c = tid % CH;   // key slot of a pass, chunk of the row
+    const int g = lane >> 2, t = lane & 3;
     const int len = prm.cache_len[b];
     const int n_tiles = (len + T - 1) / T;
     const int per_split = (n_tiles + prm.n_splits - 1) / prm.n_splits;
@@ -99,7 +125,8 @@ decode_kernel(const DecodeParams prm) {
     __shared__ __align__(16) uint32_t qh[R][D / 2];   // query rows, FP16 pairs (FP16 route)
     __shared__ __align__(16) uint32_t q8w[R][D / 4];  // quantised query rows, 4 bytes per word (INT8 route)
     __shared__ float dq_s[R];
-    __shared__ float S[2][R][T];               // scores, then probabilities with delta_V folded in
+    __shared__ float S[2][R][T];                      // scores (log2 domain)
+    __shared__ __align__(4) __half Ph[2][R][T + 8];   // probabilities x delta_V, FP16 (rows padded: banks)
     __shared__ float alpha_s[2][R];
     __shared__ __align__(8) uint64_t full_bar[kStages];
 
@@ -109,7 +136,7 @@ decode_kernel(const DecodeParams prm) {
         ptx::fence_mbar_init();
     }
 
-    // ---- the query rows of this KV head: FP32 copy and blockwise INT8 (block = the row) ----------
+    // ---- the query rows of this KV head: FP16 copy and blockwise INT8 (block = the row) ----------
     if (warp < R) {
         const int hq = hk * R + warp;
         const __half* qrow = prm.q + (static_cast<int64_t>(b) * prm.Hq + hq) * D;
@@ -147,10 +174,11 @@ decode_kernel(const DecodeParams prm) {
     const float* dv = prm.v_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.n_blk;
     const uint32_t* wrow = prm.words != nullptr
         ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : b) * prm.Hk + hk) * prm.W : nullptr;
+    const int chunks_per_blk = prm.tile_n / T;     // chunks per scale block
     auto route_of = [&](int tile) -> bool {
         if (wrow == nullptr) return false;
-        const int g = tile / prm.G;
-        return (wrow[g >> 5] >> (g & 31)) & 1u;
+        const int grp = tile / (chunks_per_blk * prm.G);
+        return (wrow[grp >> 5] >> (grp & 31)) & 1u;
     };
     // One thread streams a tile (the K copy its group is routed to, and V8; only the rows that exist).
     auto issue = [&](int tile, int stage) {
@@ -168,16 +196,15 @@ decode_kernel(const DecodeParams prm) {
     if (tid == 0)
         for (int s = 0; s < kStages - 1 && t0 + s < t1; ++s) issue(t0 + s, s);
 
-    float2 acc[R][8];
+    // A fragments of the INT8 route: lane t's words of query row g, in the order the K words are used
+    uint32_t qa8[W8];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+    for (int wi = 0; wi < W8; ++wi) qa8[wi] = g < R ? q8w[g < R ? g : 0][4 * (t + 4 * (wi / 4)) + (wi % 4)] : 0u;
+
+    float acc[NBLK][2];            // O~ rows g (< R), columns 2t, 2t+1 of this warp's column blocks
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[r][e] = make_float2(0.f, 0.f);
+    for (int nb = 0; nb < NBLK; ++nb) acc[nb][0] = acc[nb][1] = 0.f;
     float m_run = -INFINITY, z_run = 0.f;     // state of query row `warp` (warps < R), same in all lanes
-    // this thread's 16 columns of every quantised query row, kept in registers for the whole CTA
-    uint4 q8r[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) q8r[r] = *reinterpret_cast<const uint4*>(&q8w[r][4 * c]);
 
     for (int tile = t0; tile < t1; ++tile) {
         const int it = tile - t0;
@@ -194,62 +221,53 @@ decode_kernel(const DecodeParams prm) {
         if (tid == 0 && tile + kStages - 1 < t1) issue(tile + kStages - 1, (it + kStages - 1) % kStages);
         const uint8_t* kst = ring + stage * St::kBytes;
         const uint8_t* vst = kst + St::kK;
-        // ---- phase 1: scores of the tile (log2 domain) --------------------------------------
-        const float dkt = int8 ? dk[tile] : 0.f;
+        // ---- phase 1: scores of the tile (log2 domain); this warp's keys: 8 * NB1 * warp ... ----------
+        if (int8) {
+            const float dkt = dk[tile / chunks_per_blk];
 #pragma unroll
-        for (int kt = 0; kt < KPT; ++kt) {
-            const int key = kt * KPP + slot;
-            const int j = tile * T + key;
-            float s[R];
-            if (int8) {
-                uint4 kq = make_uint4(0u, 0u, 0u, 0u);
-                if (j < len) kq = *reinterpret_cast<const uint4*>(kst + key * D + 16 * c);
-                int dot[R];
+            for (int nb = 0; nb < NB1; ++nb) {
+                const int key0 = (warp * NB1 + nb) * 8;
+                const uint8_t* krow = kst + (key0 + g) * D;       // B column g = key key0 + g
+                uint32_t kw[W8];
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    dot[r] = __dp4a(static_cast<int>(kq.x), static_cast<int>(q8r[r].x), 0);
-                    dot[r] = __dp4a(static_cast<int>(kq.y), static_cast<int>(q8r[r].y), dot[r]);
-                    dot[r] = __dp4a(static_cast<int>(kq.z), static_cast<int>(q8r[r].z), dot[r]);
-                    dot[r] = __dp4a(static_cast<int>(kq.w), static_cast<int>(q8r[r].w), dot[r]);
+                for (int ch = 0; ch < W8 / 4; ++ch) {
+                    const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
+                    kw[4 * ch] = q.x; kw[4 * ch + 1] = q.y; kw[4 * ch + 2] = q.z; kw[4 * ch + 3] = q.w;
                 }
+                int c[4] = {0, 0, 0, 0};
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-#pragma unroll
-                    for (int o = CH / 2; o > 0; o >>= 1) dot[r] += __shfl_xor_sync(0xffffffffu, dot[r], o);
-                    s[r] = static_cast<float>(dot[r]) * (prm.scale_log2 * dq_s[r] * dkt);
-                }
-            } else {
-                uint4 k0 = make_uint4(0u, 0u, 0u, 0u), k1 = k0;
-                if (j < len) {
-                    const uint4* src = reinterpret_cast<const uint4*>(kst + (key * D + 16 * c) * 2);
-                    k0 = src[0];
-                    k1 = src[1];
-                }
-                const uint32_t kw[8] = {k0.x, k0.y, k0.z, k0.w, k1.x, k1.y, k1.z, k1.w};
-                float2 kf[8];
-#pragma unroll
-                for (int w = 0; w < 8; ++w) kf[w] = __half22float2(*reinterpret_cast<const __half2*>(&kw[w]));
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    // this thread's 16 columns of query row r (two 16-byte reads, the same for every key)
-                    const uint4 qa = *reinterpret_cast<const uint4*>(&qh[r][8 * c]);
-                    const uint4 qb = *reinterpret_cast<const uint4*>(&qh[r][8 * c + 4]);
-                    const uint32_t qw[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
-                    float dot = 0.f;
-#pragma unroll
-                    for (int w = 0; w < 8; ++w) {
-                        const float2 qv = __half22float2(*reinterpret_cast<const __half2*>(&qw[w]));
-                        dot = fmaf(kf[w].x, qv.x, dot);
-                        dot = fmaf(kf[w].y, qv.y, dot);
-                    }
-#pragma unroll
-                    for (int o = CH / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    s[r] = dot * prm.scale_log2;
+                for (int ks = 0; ks < W8 / 2; ++ks) mma_s8(c, qa8[2 * ks], qa8[2 * ks + 1], kw[2 * ks], kw[2 * ks + 1]);
+                if (g < R) {
+                    const float a = prm.scale_log2 * dq_s[g] * dkt;
+                    const int j = tile * T + key0 + 2 * t;
+                    S[buf][g][key0 + 2 * t] = j < len ? static_cast<float>(c[0]) * a : -INFINITY;
+                    S[buf][g][key0 + 2 * t + 1] = j + 1 < len ? static_cast<float>(c[1]) * a : -INFINITY;
                 }
             }
-            if (c == 0) {
+        } else {
+            uint32_t qa16[W16];
 #pragma unroll
-                for (int r = 0; r < R; ++r) S[buf][r][key] = j < len ? s[r] : -INFINITY;
+            for (int ch = 0; ch < W16 / 4; ++ch) {
+                uint4 q = make_uint4(0u, 0u, 0u, 0u);
+                if (g < R) q = *reinterpret_cast<const uint4*>(&qh[g < R ? g : 0][4 * (t + 4 * ch)]);
+                qa16[4 * ch] = q.x; qa16[4 * ch + 1] = q.y; qa16[4 * ch + 2] = q.z; qa16[4 * ch + 3] = q.w;
+            }
+#pragma unroll
+            for (int nb = 0; nb < NB1; ++nb) {
+                const int key0 = (warp * NB1 + nb) * 8;
+                const uint8_t* krow = kst + (key0 + g) * D * 2;
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ch = 0; ch < W16 / 4; ++ch) {
+                    const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
+                    mma_f16(c, qa16[4 * ch], qa16[4 * ch + 1], q.x, q.y);
+                    mma_f16(c, qa16[4 * ch + 2], qa16[4 * ch + 3], q.z, q.w);
+                }
+                if (g < R) {
+                    const int j = tile * T + key0 + 2 * t;
+                    S[buf][g][key0 + 2 * t] = j < len ? c[0] * prm.scale_log2 : -INFINITY;
+                    S[buf][g][key0 + 2 * t + 1] = j + 1 < len ? c[1] * prm.scale_log2 : -INFINITY;
+                }
             }
         }
         __syncthreads();
@@ -266,13 +284,13 @@ decode_kernel(const DecodeParams prm) {
             for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
             const float m_new = fmaxf(m_run, tmax);       // finite: the tile holds at least one key
             const float alpha = exp2f(m_run - m_new);     // 0 on the first tile
-            const float dvt = dv[tile];
+            const float dvt = dv[tile / chunks_per_blk];
             float sum = 0.f;
 #pragma unroll
             for (int x = 0; x < T / 32; ++x) {
                 const float p = exp2f(sv[x] - m_new);
                 sum += p;
-                S[buf][warp][lane + 32 * x] = round_to_half(p * dvt);
+                Ph[buf][warp][lane + 32 * x] = __float2half_rn(p * dvt);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -281,64 +299,88 @@ decode_kernel(const DecodeParams prm) {
             if (lane == 0) alpha_s[buf][warp] = alpha;
         }
         __syncthreads();
-        // ---- phase 3: O~ = alpha * O~ + P V8 over this thread's keys and 16 columns ----------------
+        // ---- phase 3: O~ = alpha * O~ + P V8 over this warp's 16 keys and column blocks ----------------
+        {
+            const int ks = warp / NSPLIT, nb0 = (warp % NSPLIT) * NBLK;
+            const float al = g < R ? alpha_s[buf][g < R ? g : 0] : 1.f;
+            if (__any_sync(0xffffffffu, al != 1.f)) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const float a = alpha_s[buf][r];     // the same for the whole CTA; 1 unless the maximum moved
-            if (a != 1.f) {
-                const float2 a2 = make_float2(a, a);
+                for (int nb = 0; nb < NBLK; ++nb) { acc[nb][0] *= al; acc[nb][1] *= al; }
+            }
+            uint32_t pa0 = 0u, pa2 = 0u;
+            if (g < R) {
+                pa0 = *reinterpret_cast<const uint32_t*>(&Ph[buf][g][16 * ks + 2 * t]);
+                pa2 = *reinterpret_cast<const uint32_t*>(&Ph[buf][g][16 * ks + 2 * t + 8]);
+            }
+            // the four cached rows whose pairs this lane feeds: keys 2t, 2t+1 and 2t+8, 2t+9 of the step,
+            // BPG bytes each, at this lane group's columns of this warp's blocks
+            const uint8_t* vbase = vst + (16 * ks + 2 * t) * D + BPG * g + nb0;
+            uint32_t u[4][NBLK / 4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[r][e] = __fmul2_rn(acc[r][e], a2);
+            for (int r4 = 0; r4 < 4; ++r4) {
+                const uint8_t* src = vbase + ((r4 & 1) + (r4 >> 1) * 8) * D;
+                if constexpr (NBLK == 16) {
+                    const uint4 q = *reinterpret_cast<const uint4*>(src);
+                    u[r4][0] = q.x; u[r4][1] = q.y; u[r4][2] = q.z; u[r4][3] = q.w;
+                } else if constexpr (NBLK == 8) {
+                    const uint2 q = *reinterpret_cast<const uint2*>(src);
+                    u[r4][0] = q.x; u[r4][1] = q.y;
+                } else {
+                    u[r4][0] = *reinterpret_cast<const uint32_t*>(src);
+                }
+#pragma unroll
+                for (int w = 0; w < NBLK / 4; ++w) u[r4][w] ^= 0x80808080u;   // signed -> offset binary
+            }
+            const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+            float dummy[2] = {0.f, 0.f};
+#pragma unroll
+            for (int w = 0; w < NBLK / 4; ++w) {
+                // bytes of rows (k0, k1) and (k2, k3) interleaved: {k0[e], k1[e]} pairs for e = 0..3
+                const uint32_t lo01 = __byte_perm(u[0][w], u[1][w], 0x5140), hi01 = __byte_perm(u[0][w], u[1][w], 0x7362);
+                const uint32_t lo23 = __byte_perm(u[2][w], u[3][w], 0x5140), hi23 = __byte_perm(u[2][w], u[3][w], 0x7362);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t s01 = e < 2 ? lo01 : hi01, s23 = e < 2 ? lo23 : hi23;
+                    const uint32_t sel = (e & 1) ? 0x4342u : 0x4140u;
+                    // half2(1024 + (x + 128)) - 1152 = half2(x), exactly
+                    uint32_t b0 = __byte_perm(s01, 0x64646464u, sel), b1 = __byte_perm(s23, 0x64646464u, sel);
+                    const __half2 h0 = __hsub2(*reinterpret_cast<const __half2*>(&b0), off);
+                    const __half2 h1 = __hsub2(*reinterpret_cast<const __half2*>(&b1), off);
+                    float c[4] = {acc[4 * w + e][0], acc[4 * w + e][1], dummy[0], dummy[1]};
+                    mma_f16(c, pa0, pa2, *reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    acc[4 * w + e][0] = c[0]; acc[4 * w + e][1] = c[1];
+                    dummy[0] = c[2]; dummy[1] = c[3];
+                }
             }
         }
-#pragma unroll
-        for (int kt = 0; kt < KPT; ++kt) {
-            const int key = kt * KPP + slot;
-            if (tile * T + key >= len) continue;       // rows that were not copied
-            const uint4 vq = *reinterpret_cast<const uint4*>(vst + key * D + 16 * c);
-            const uint32_t vw[4] = {vq.x, vq.y, vq.z, vq.w};
-            float2 vf[8];
-#pragma unroll
-            for (int w = 0; w < 4; ++w) bytes_to_floats(vw[w], *reinterpret_cast<float2(*)[2]>(&vf[2 * w]));
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const float p = S[buf][r][key];
-                const float2 pp = make_float2(p, p);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[r][e] = __ffma2_rn(vf[e], pp, acc[r][e]);
-            }
-        }
-        // the next tile writes the other score buffer; the sync at its top orders the reuse of the stage
+        // the next tile writes the other score buffers; the sync at its top orders the reuse of the stage
     }
 
-    // ---- partial result of this split: sum over the key slots, then (m, z, O~) to the workspace -----
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-#pragma unroll
-            for (int o = CH; o < 32; o <<= 1) {
-                acc[r][e].x += __shfl_xor_sync(0xffffffffu, acc[r][e].x, o);
-                acc[r][e].y += __shfl_xor_sync(0xffffffffu, acc[r][e].y, o);
-            }
-        }
+    // ---- partial result of this split: sum over the warps (key steps), then (m, z, O~) to the workspace ----
     __syncthreads();   // every thread is done with the ring: reuse it for the reduction over the warps
     float (*red)[R][D] = reinterpret_cast<float (*)[R][D]>(ring);
-    if (lane < CH) {
+    {
+        const int nb0 = (warp % NSPLIT) * NBLK;
+        if constexpr (NSPLIT > 1) {
+            // warps of one key step hold disjoint column blocks: zero the rest of this warp's plane first
+            for (int idx = lane; idx < R * D; idx += 32) red[warp][idx / D][idx % D] = 0.f;
+            __syncwarp();
+        }
+        if (g < R) {
 #pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                red[warp][r][16 * lane + 2 * e] = acc[r][e].x;
-                red[warp][r][16 * lane + 2 * e + 1] = acc[r][e].y;
+            for (int nb = 0; nb < NBLK; ++nb) {
+                // column n of block nb is d = (D/8) n + nb; this lane holds n = 2t, 2t+1
+                red[warp][g][BPG * (2 * t) + nb0 + nb] = acc[nb][0];
+                red[warp][g][BPG * (2 * t + 1) + nb0 + nb] = acc[nb][1];
             }
+        }
     }
     __syncthreads();
     for (int idx = tid; idx < R * D; idx += kThreads) {
         const int r = idx / D, e = idx - r * D;
         float o = 0.f;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) o += red[w][r][e];
+        for (int w = 0; w < kWarps; ++w) o += red[w][r][e];
         const int64_t row = (static_cast<int64_t>(b) * prm.Hq + hk * R + r) * prm.n_splits + split;
         prm.o_part[row * D + e] = o;
     }
@@ -471,6 +513,7 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     DecodeParams prm{};
     prm.B = p->batch; prm.Hq = p->heads_q; prm.Hk = p->heads_kv; prm.max_len = p->max_len; prm.G = p->group;
     prm.nb = p->mask_batch; prm.W = g.W; prm.n_splits = g.n_splits; prm.n_blk = g.n_blk;
+    prm.tile_n = p->tile_n;
     const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
     prm.scale_log2 = scale * kLog2e;
     prm.q = static_cast<const __half*>(q_f16);
@@ -486,6 +529,8 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int R = p->heads_q / p->heads_kv;
     __half* out = static_cast<__half*>(out_f16);
+    // keys are streamed and processed one routing tile at a time (64-key chunks with a deeper ring
+    // were slower: the per-chunk barriers cost more than the extra bytes in flight gain)
     if (p->head_dim == 128 && p->tile_n == 128) return launch_r<128, 128>(R, prm, out, lse, s);
     if (p->head_dim == 128 && p->tile_n == 64) return launch_r<128, 64>(R, prm, out, lse, s);
     if (p->head_dim == 64 && p->tile_n == 128) return launch_r<64, 128>(R, prm, out, lse, s);
