@@ -52,7 +52,12 @@ __device__ __forceinline__ void bytes_to_floats(uint32_t w, float2 (&f)[2]) {
                                   __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653))), bias);
 }
 
-constexpr int kStages = 2;                 // ring of key/value chunks in shared memory
+#ifndef TILEMIX_DECODE_STAGES
+#define TILEMIX_DECODE_STAGES 2
+#define TILEMIX_DECODE_CHUNK 128
+#endif
+constexpr int kStages = TILEMIX_DECODE_STAGES;   // ring of key/value tiles in shared memory
+constexpr int kChunk = TILEMIX_DECODE_CHUNK;     // keys per kernel tile when tile_n allows it
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 
 template <int D, int T>
@@ -61,17 +66,6 @@ struct Stage {
     static constexpr int kV = T * D;
     static constexpr int kBytes = kK + kV;
 };
-
-// Bounded wait on a "tile landed" barrier; false when the time limit ran out.
-__device__ __forceinline__ bool wait_tile(uint32_t bar, uint32_t parity) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = ptx::globaltimer_ns();
-    uint32_t it = 0;
-    while (!ptx::mbar_try_wait(bar, parity)) {
-        if ((++it & 63u) == 0u && ptx::globaltimer_ns() - t0 > kTimeoutNs) return false;
-    }
-    return true;
-}
 
 // ---- warp-level tensor-core MMAs (m16n8k32 INT8 / m16n8k16 FP16, FP32 or INT32 accumulators) ----------
 // Lane l holds, with g = l / 4 and t = l % 4: A rows g (a0, a2) and g + 8 (a1, a3), B column g, C rows g
@@ -88,31 +82,36 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a2,
                  : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
-// D: head dim; R: query heads per KV head; T: keys per chunk (the scale block / routing tile tile_n is a
-// multiple of it).  Chunks are contiguous in the cache, so one thread streams them into a ring of
-// shared-memory stages with untiled bulk copies, kStages - 1 chunks ahead of their use; with two CTAs
-// per SM this keeps 100-150 KB per SM in flight.  Per chunk:
-//  (1) scores S[R x T] = Q K^T on the tensor cores, the R query rows being rows 0..R-1 of a 16-row A
-//      operand; each warp takes T/8 keys.  The contraction index may be permuted freely as long as Q and K
-//      use the same permutation, so lane t simply takes the 16-byte chunks t, t+4, ... of a row.
-//  (2) the online softmax of each query row by one warp; P gets delta_V and is rounded to FP16.
-//  (3) O~[R x D] += P V8 on the tensor cores; each warp takes 16 keys (T = 128) and all columns.  V8 is
-//      converted to FP16 in registers (exactly); the output columns are permuted (column n of block nb
-//      is d = (D/8) n + nb) so that the bytes a lane needs from a cached row are contiguous.
+// D: head dim; R: query heads per KV head; T: keys per tile (= scale block = routing tile).
+// Tiles are contiguous in the cache, so they are streamed into a ring of shared-memory stages with
+// untiled bulk copies ("full" / "empty" mbarriers per stage), issued by one lane of the last warp
+// before it turns to its own share of a tile.  The eight warps never synchronise with one another
+// inside the loop: each one owns 16 keys of every tile (and, for
+// 64-key tiles, half of the output columns) and runs its own flash-decoding recurrence on them --
+//  (1) scores S[R x 16] = Q K^T on the tensor cores, the R query rows being rows 0..R-1 of a 16-row A
+//      operand.  The contraction index may be permuted freely as long as Q and K use the same
+//      permutation, so lane t simply takes the 16-byte chunks t, t+4, ... of a row;
+//  (2) running maximum and sum of its own keys (two shuffles per row), P = 2^(s - m) times delta_V,
+//      rounded to FP16 -- the score fragment is already laid out as the A operand of the next product;
+//  (3) O~[R x D] += P V8 on the tensor cores.  V8 is converted to FP16 in registers (exactly); the
+//      output columns are permuted (column n of block nb is d = (D/8) n + nb) so that the bytes a
+//      lane needs from a cached row are contiguous.
+// After the loop the eight (m, z, O~) are merged in shared memory like splits.
+constexpr int kConsumerWarps = 8;
+constexpr int kDecodeThreads = kConsumerWarps * 32;   // 2 CTAs/SM = 4 warps per scheduler: 128 registers each
+
 template <int D, int R, int T>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kDecodeThreads, 2)
 decode_kernel(const DecodeParams prm) {
     using St = Stage<D, T>;
-    constexpr int kWarps = kThreads / 32;
-    constexpr int NB1 = T / 8 / kWarps;           // key blocks (8 keys) per warp in phase 1
     constexpr int W8 = D / 16, W16 = D / 8;       // 32-bit words per lane and row: INT8 / FP16 operand
-    constexpr int KS3 = T / 16;                   // 16-key steps of a tile in phase 3
-    constexpr int NSPLIT = kWarps / KS3;          // warps sharing one such step (each takes some column blocks)
-    constexpr int NBLK = D / 8 / NSPLIT;          // column blocks per warp in phase 3
+    constexpr int KS3 = T / 16;                   // 16-key steps of a tile
+    constexpr int NSPLIT = kConsumerWarps / KS3;  // warps sharing one step (each takes some column blocks)
+    constexpr int NBLK = D / 8 / NSPLIT;          // column blocks per warp
     constexpr int BPG = D / 8;                    // bytes of a cached V row per lane group
-    static_assert(NB1 >= 1 && KS3 <= kWarps && kWarps % KS3 == 0, "tile shape vs warps");
-    static_assert(kStages * St::kBytes >= static_cast<int>(kWarps * R * D * sizeof(float)),
-                  "the final reduction reuses the ring");
+    static_assert(KS3 <= kConsumerWarps && kConsumerWarps % KS3 == 0, "tile shape vs warps");
+    static_assert(kStages * St::kBytes >= static_cast<int>(kConsumerWarps * R * (D + 2) * sizeof(float)),
+                  "the final merge reuses the ring");
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -125,14 +124,16 @@ decode_kernel(const DecodeParams prm) {
     __shared__ __align__(16) uint32_t qh[R][D / 2];   // query rows, FP16 pairs (FP16 route)
     __shared__ __align__(16) uint32_t q8w[R][D / 4];  // quantised query rows, 4 bytes per word (INT8 route)
     __shared__ float dq_s[R];
-    __shared__ float S[2][R][T];                      // scores (log2 domain)
-    __shared__ __align__(4) __half Ph[2][R][T + 8];   // probabilities x delta_V, FP16 (rows padded: banks)
-    __shared__ float alpha_s[2][R];
-    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
+    __shared__ int abort_flag;
 
     const uint32_t ring_u32 = ptx::smem_u32(ring);
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), kConsumerWarps);
+        }
+        abort_flag = 0;
         ptx::fence_mbar_init();
     }
 
@@ -167,22 +168,52 @@ decode_kernel(const DecodeParams prm) {
     }
 
     const int64_t row_base = (static_cast<int64_t>(b) * prm.Hk + hk) * prm.max_len;
-    const int8_t* k8 = prm.k8 + row_base * D;
-    const int8_t* v8 = prm.v8 + row_base * D;
-    const __half* k16 = prm.k16 != nullptr ? prm.k16 + row_base * D : nullptr;
     const float* dk = prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.n_blk;
     const float* dv = prm.v_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.n_blk;
     const uint32_t* wrow = prm.words != nullptr
         ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : b) * prm.Hk + hk) * prm.W : nullptr;
-    const int chunks_per_blk = prm.tile_n / T;     // chunks per scale block
+    // the kernel's tile (T keys) may be a fraction of the scale block / routing tile tile_n
+    const int per_blk = prm.tile_n / T;
     auto route_of = [&](int tile) -> bool {
         if (wrow == nullptr) return false;
-        const int grp = tile / (chunks_per_blk * prm.G);
+        const int grp = tile / (per_blk * prm.G);
         return (wrow[grp >> 5] >> (grp & 31)) & 1u;
     };
-    // One thread streams a tile (the K copy its group is routed to, and V8; only the rows that exist).
-    auto issue = [&](int tile, int stage) {
-        const uint32_t rows = static_cast<uint32_t>(min(T, len - tile * T));
+    // Bounded wait on a ring barrier; false when the CTA is giving up.
+    auto wait_ring = [&](uint64_t* bar, uint32_t parity) -> bool {
+        const uint32_t addr = ptx::smem_u32(bar);
+        if (ptx::mbar_try_wait(addr, parity)) return true;
+        const uint64_t start = ptx::globaltimer_ns();
+        uint32_t spins = 0;
+        while (!ptx::mbar_try_wait(addr, parity)) {
+            if ((++spins & 63u) == 0u) {
+                if (*reinterpret_cast<volatile int*>(&abort_flag)) return false;
+                if (ptx::globaltimer_ns() - start > kTimeoutNs) {
+                    *reinterpret_cast<volatile int*>(&abort_flag) = 1;
+                    return false;
+                }
+            }
+        }
+        return true;
+    };
+    __syncthreads();   // barriers initialised, query rows staged
+
+    // per-warp flash-decoding state: rows g (< R) of this warp's keys
+    float m_run = -INFINITY, z_part = 0.f;          // z_part: this lane's share of the row sum
+    float acc[NBLK][2];                             // O~ rows g, columns 2t, 2t+1 of this warp's blocks
+#pragma unroll
+    for (int nb = 0; nb < NBLK; ++nb) acc[nb][0] = acc[nb][1] = 0.f;
+
+    // Refill of the ring by one lane (of the last warp): tile `tile` into its stage, after every warp
+    // has handed that stage back.  Returns false when the CTA is giving up.
+    const int8_t* k8 = prm.k8 + row_base * D;
+    const int8_t* v8 = prm.v8 + row_base * D;
+    const __half* k16 = prm.k16 != nullptr ? prm.k16 + row_base * D : nullptr;
+    auto produce = [&](int tile) -> bool {
+        const int it = tile - t0, stage = it % kStages;
+        // the first pass over the ring finds every stage free
+        if (it >= kStages && !wait_ring(&empty_bar[stage], ((it / kStages) - 1) & 1)) return false;
+        const uint32_t rows = static_cast<uint32_t>(min(T, len - tile * T));   // only rows that exist
         const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
         const uint32_t dst = ring_u32 + stage * St::kBytes;
         const bool int8 = route_of(tile);
@@ -191,174 +222,152 @@ decode_kernel(const DecodeParams prm) {
         if (int8) ptx::bulk_load_1d(dst, k8 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
         else ptx::bulk_load_1d(dst, k16 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
         ptx::bulk_load_1d(dst + St::kK, v8 + static_cast<int64_t>(tile) * T * D, rows * D, bar);
+        return true;
     };
-    __syncthreads();   // barriers initialised, query rows staged
-    if (tid == 0)
-        for (int s = 0; s < kStages - 1 && t0 + s < t1; ++s) issue(t0 + s, s);
+    const bool producer = warp == kConsumerWarps - 1 && lane == 0;
+    if (producer)
+        for (int s = 0; s < kStages - 1 && t0 + s < t1; ++s) produce(t0 + s);
+    {
+        // ================================================================ consumers
+        const int ks = warp / NSPLIT, nb0 = (warp % NSPLIT) * NBLK;   // this warp's keys and column blocks
+        const bool counts_z = (warp % NSPLIT) == 0;                    // one warp per key step sums z
+        // A fragments of the INT8 route: lane t's words of query row g, in the order the K words are used
+        uint32_t qa8[W8];
+#pragma unroll
+        for (int wi = 0; wi < W8; ++wi) qa8[wi] = g < R ? q8w[g < R ? g : 0][4 * (t + 4 * (wi / 4)) + (wi % 4)] : 0u;
+        const float dq = g < R ? dq_s[g < R ? g : 0] : 0.f;
 
-    // A fragments of the INT8 route: lane t's words of query row g, in the order the K words are used
-    uint32_t qa8[W8];
+        for (int tile = t0; tile < t1; ++tile) {
+            const int it = tile - t0, stage = it % kStages;
+            if (producer && tile + kStages - 1 < t1) produce(tile + kStages - 1);   // keeps the ring full
+            const bool int8 = route_of(tile);
+            // ahead of the wait (fetching them a tile ahead instead costs registers and was slower)
+            const float dkt = int8 ? dk[tile / per_blk] : 0.f, dvt = dv[tile / per_blk];
+            if (!wait_ring(&full_bar[stage], (it / kStages) & 1)) break;
+            const uint8_t* kst = ring + stage * St::kBytes;
+            const uint8_t* vst = kst + St::kK;
+            // ---- (1) scores of this warp's 16 keys, rows g: s[nb][0..1] = keys 8 nb + 2t, 2t + 1 ----------
+            float sc[2][2];
+            if (int8) {
+                const float a = prm.scale_log2 * dq * dkt;
 #pragma unroll
-    for (int wi = 0; wi < W8; ++wi) qa8[wi] = g < R ? q8w[g < R ? g : 0][4 * (t + 4 * (wi / 4)) + (wi % 4)] : 0u;
-
-    float acc[NBLK][2];            // O~ rows g (< R), columns 2t, 2t+1 of this warp's column blocks
+                for (int nb = 0; nb < 2; ++nb) {
+                    const uint8_t* krow = kst + (16 * ks + 8 * nb + g) * D;       // B column g = that key
+                    uint32_t kw[W8];
 #pragma unroll
-    for (int nb = 0; nb < NBLK; ++nb) acc[nb][0] = acc[nb][1] = 0.f;
-    float m_run = -INFINITY, z_run = 0.f;     // state of query row `warp` (warps < R), same in all lanes
-
-    for (int tile = t0; tile < t1; ++tile) {
-        const int it = tile - t0;
-        const int buf = it & 1, stage = it % kStages;
-        const bool int8 = route_of(tile);
-        const bool landed = wait_tile(ptx::smem_u32(&full_bar[stage]), (it / kStages) & 1);
-        // Everyone is past the previous tile here, so its stage can be refilled.
-        if (__syncthreads_or(!landed)) {
-            if (tid == 0 && atomicCAS(&prm.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
-                prm.status[1] = 16; prm.status[2] = tile; prm.status[3] = 0;
-            }
-            return;   // no copy of this CTA is known to be in flight into a stage it would still read
-        }
-        if (tid == 0 && tile + kStages - 1 < t1) issue(tile + kStages - 1, (it + kStages - 1) % kStages);
-        const uint8_t* kst = ring + stage * St::kBytes;
-        const uint8_t* vst = kst + St::kK;
-        // ---- phase 1: scores of the tile (log2 domain); this warp's keys: 8 * NB1 * warp ... ----------
-        if (int8) {
-            const float dkt = dk[tile / chunks_per_blk];
+                    for (int ch = 0; ch < W8 / 4; ++ch) {
+                        const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
+                        kw[4 * ch] = q.x; kw[4 * ch + 1] = q.y; kw[4 * ch + 2] = q.z; kw[4 * ch + 3] = q.w;
+                    }
+                    int c[4] = {0, 0, 0, 0};
 #pragma unroll
-            for (int nb = 0; nb < NB1; ++nb) {
-                const int key0 = (warp * NB1 + nb) * 8;
-                const uint8_t* krow = kst + (key0 + g) * D;       // B column g = key key0 + g
-                uint32_t kw[W8];
-#pragma unroll
-                for (int ch = 0; ch < W8 / 4; ++ch) {
-                    const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
-                    kw[4 * ch] = q.x; kw[4 * ch + 1] = q.y; kw[4 * ch + 2] = q.z; kw[4 * ch + 3] = q.w;
+                    for (int k = 0; k < W8 / 2; ++k) mma_s8(c, qa8[2 * k], qa8[2 * k + 1], kw[2 * k], kw[2 * k + 1]);
+                    sc[nb][0] = static_cast<float>(c[0]) * a;
+                    sc[nb][1] = static_cast<float>(c[1]) * a;
                 }
-                int c[4] = {0, 0, 0, 0};
-#pragma unroll
-                for (int ks = 0; ks < W8 / 2; ++ks) mma_s8(c, qa8[2 * ks], qa8[2 * ks + 1], kw[2 * ks], kw[2 * ks + 1]);
-                if (g < R) {
-                    const float a = prm.scale_log2 * dq_s[g] * dkt;
-                    const int j = tile * T + key0 + 2 * t;
-                    S[buf][g][key0 + 2 * t] = j < len ? static_cast<float>(c[0]) * a : -INFINITY;
-                    S[buf][g][key0 + 2 * t + 1] = j + 1 < len ? static_cast<float>(c[1]) * a : -INFINITY;
-                }
-            }
-        } else {
-            uint32_t qa16[W16];
-#pragma unroll
-            for (int ch = 0; ch < W16 / 4; ++ch) {
-                uint4 q = make_uint4(0u, 0u, 0u, 0u);
-                if (g < R) q = *reinterpret_cast<const uint4*>(&qh[g < R ? g : 0][4 * (t + 4 * ch)]);
-                qa16[4 * ch] = q.x; qa16[4 * ch + 1] = q.y; qa16[4 * ch + 2] = q.z; qa16[4 * ch + 3] = q.w;
-            }
-#pragma unroll
-            for (int nb = 0; nb < NB1; ++nb) {
-                const int key0 = (warp * NB1 + nb) * 8;
-                const uint8_t* krow = kst + (key0 + g) * D * 2;
-                float c[4] = {0.f, 0.f, 0.f, 0.f};
+            } else {
+                uint32_t qa16[W16];
 #pragma unroll
                 for (int ch = 0; ch < W16 / 4; ++ch) {
-                    const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
-                    mma_f16(c, qa16[4 * ch], qa16[4 * ch + 1], q.x, q.y);
-                    mma_f16(c, qa16[4 * ch + 2], qa16[4 * ch + 3], q.z, q.w);
+                    uint4 q = make_uint4(0u, 0u, 0u, 0u);
+                    if (g < R) q = *reinterpret_cast<const uint4*>(&qh[g < R ? g : 0][4 * (t + 4 * ch)]);
+                    qa16[4 * ch] = q.x; qa16[4 * ch + 1] = q.y; qa16[4 * ch + 2] = q.z; qa16[4 * ch + 3] = q.w;
                 }
-                if (g < R) {
-                    const int j = tile * T + key0 + 2 * t;
-                    S[buf][g][key0 + 2 * t] = j < len ? c[0] * prm.scale_log2 : -INFINITY;
-                    S[buf][g][key0 + 2 * t + 1] = j + 1 < len ? c[1] * prm.scale_log2 : -INFINITY;
+#pragma unroll
+                for (int nb = 0; nb < 2; ++nb) {
+                    const uint8_t* krow = kst + (16 * ks + 8 * nb + g) * D * 2;
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int ch = 0; ch < W16 / 4; ++ch) {
+                        const uint4 q = *reinterpret_cast<const uint4*>(krow + 16 * (t + 4 * ch));
+                        mma_f16(c, qa16[4 * ch], qa16[4 * ch + 1], q.x, q.y);
+                        mma_f16(c, qa16[4 * ch + 2], qa16[4 * ch + 3], q.z, q.w);
+                    }
+                    sc[nb][0] = c[0] * prm.scale_log2;
+                    sc[nb][1] = c[1] * prm.scale_log2;
                 }
             }
-        }
-        __syncthreads();
-        // ---- phase 2: online softmax of query row `warp`; P gets delta_V and is rounded to FP16 ----
-        if (warp < R) {
-            float sv[T / 32];
-            float tmax = -INFINITY;
+            // keys beyond the cached length (stale shared memory) do not exist
+            const int j0 = tile * T + 16 * ks + 2 * t;
 #pragma unroll
-            for (int x = 0; x < T / 32; ++x) {
-                sv[x] = S[buf][warp][lane + 32 * x];
-                tmax = fmaxf(tmax, sv[x]);
+            for (int nb = 0; nb < 2; ++nb) {
+                if (j0 + 8 * nb >= len) sc[nb][0] = -INFINITY;
+                if (j0 + 8 * nb + 1 >= len) sc[nb][1] = -INFINITY;
             }
+            // ---- (2) this warp's online softmax over its own keys ------------------------------------------
+            float tmax = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+            const float m_new = fmaxf(m_run, tmax);
+            // a warp whose 16 keys of this tile all lie beyond the cache keeps its state (m_new may be -inf)
+            const float m_use = m_new == -INFINITY ? 0.f : m_new;
+            const float alpha = exp2f(m_run - m_use);        // 0 on the first keys, 1 if the maximum stands
+            float p[2][2];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-            const float m_new = fmaxf(m_run, tmax);       // finite: the tile holds at least one key
-            const float alpha = exp2f(m_run - m_new);     // 0 on the first tile
-            const float dvt = dv[tile / chunks_per_blk];
-            float sum = 0.f;
-#pragma unroll
-            for (int x = 0; x < T / 32; ++x) {
-                const float p = exp2f(sv[x] - m_new);
-                sum += p;
-                Ph[buf][warp][lane + 32 * x] = __float2half_rn(p * dvt);
+            for (int nb = 0; nb < 2; ++nb) {
+                p[nb][0] = exp2f(sc[nb][0] - m_use);
+                p[nb][1] = exp2f(sc[nb][1] - m_use);
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            z_run = z_run * alpha + sum;
+            z_part = z_part * alpha + ((p[0][0] + p[0][1]) + (p[1][0] + p[1][1]));
             m_run = m_new;
-            if (lane == 0) alpha_s[buf][warp] = alpha;
-        }
-        __syncthreads();
-        // ---- phase 3: O~ = alpha * O~ + P V8 over this warp's 16 keys and column blocks ----------------
-        {
-            const int ks = warp / NSPLIT, nb0 = (warp % NSPLIT) * NBLK;
-            const float al = g < R ? alpha_s[buf][g < R ? g : 0] : 1.f;
-            if (__any_sync(0xffffffffu, al != 1.f)) {
+            if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
-                for (int nb = 0; nb < NBLK; ++nb) { acc[nb][0] *= al; acc[nb][1] *= al; }
+                for (int nb = 0; nb < NBLK; ++nb) { acc[nb][0] *= alpha; acc[nb][1] *= alpha; }
             }
-            uint32_t pa0 = 0u, pa2 = 0u;
-            if (g < R) {
-                pa0 = *reinterpret_cast<const uint32_t*>(&Ph[buf][g][16 * ks + 2 * t]);
-                pa2 = *reinterpret_cast<const uint32_t*>(&Ph[buf][g][16 * ks + 2 * t + 8]);
-            }
+            // P x delta_V, FP16: the score fragment (row g, keys 2t, 2t+1 of each 8-key block) is the A
+            // fragment of the PV product over these 16 keys
+            const __half2 h0 = __floats2half2_rn(p[0][0] * dvt, p[0][1] * dvt);
+            const __half2 h2 = __floats2half2_rn(p[1][0] * dvt, p[1][1] * dvt);
+            const uint32_t pa0 = g < R ? *reinterpret_cast<const uint32_t*>(&h0) : 0u;
+            const uint32_t pa2 = g < R ? *reinterpret_cast<const uint32_t*>(&h2) : 0u;
+            // ---- (3) O~ += P V8 ------------------------------------------------------------------------------
             // the four cached rows whose pairs this lane feeds: keys 2t, 2t+1 and 2t+8, 2t+9 of the step,
-            // BPG bytes each, at this lane group's columns of this warp's blocks
+            // at this lane group's columns of this warp's blocks
             const uint8_t* vbase = vst + (16 * ks + 2 * t) * D + BPG * g + nb0;
-            uint32_t u[4][NBLK / 4];
-#pragma unroll
-            for (int r4 = 0; r4 < 4; ++r4) {
-                const uint8_t* src = vbase + ((r4 & 1) + (r4 >> 1) * 8) * D;
-                if constexpr (NBLK == 16) {
-                    const uint4 q = *reinterpret_cast<const uint4*>(src);
-                    u[r4][0] = q.x; u[r4][1] = q.y; u[r4][2] = q.z; u[r4][3] = q.w;
-                } else if constexpr (NBLK == 8) {
-                    const uint2 q = *reinterpret_cast<const uint2*>(src);
-                    u[r4][0] = q.x; u[r4][1] = q.y;
-                } else {
-                    u[r4][0] = *reinterpret_cast<const uint32_t*>(src);
-                }
-#pragma unroll
-                for (int w = 0; w < NBLK / 4; ++w) u[r4][w] ^= 0x80808080u;   // signed -> offset binary
-            }
             const __half2 off = __floats2half2_rn(1152.f, 1152.f);
             float dummy[2] = {0.f, 0.f};
 #pragma unroll
             for (int w = 0; w < NBLK / 4; ++w) {
+                // four column blocks at a time: one 32-bit word of each of the four rows
+                uint32_t u[4];
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4)
+                    u[r4] = *reinterpret_cast<const uint32_t*>(vbase + ((r4 & 1) + (r4 >> 1) * 8) * D + 4 * w) ^ 0x80808080u;
+                if (w == NBLK / 4 - 1) {
+                    // last read of this stage by this warp: hand the stage back
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&empty_bar[stage]));
+                }
                 // bytes of rows (k0, k1) and (k2, k3) interleaved: {k0[e], k1[e]} pairs for e = 0..3
-                const uint32_t lo01 = __byte_perm(u[0][w], u[1][w], 0x5140), hi01 = __byte_perm(u[0][w], u[1][w], 0x7362);
-                const uint32_t lo23 = __byte_perm(u[2][w], u[3][w], 0x5140), hi23 = __byte_perm(u[2][w], u[3][w], 0x7362);
+                const uint32_t lo01 = __byte_perm(u[0], u[1], 0x5140), hi01 = __byte_perm(u[0], u[1], 0x7362);
+                const uint32_t lo23 = __byte_perm(u[2], u[3], 0x5140), hi23 = __byte_perm(u[2], u[3], 0x7362);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const uint32_t s01 = e < 2 ? lo01 : hi01, s23 = e < 2 ? lo23 : hi23;
                     const uint32_t sel = (e & 1) ? 0x4342u : 0x4140u;
                     // half2(1024 + (x + 128)) - 1152 = half2(x), exactly
                     uint32_t b0 = __byte_perm(s01, 0x64646464u, sel), b1 = __byte_perm(s23, 0x64646464u, sel);
-                    const __half2 h0 = __hsub2(*reinterpret_cast<const __half2*>(&b0), off);
-                    const __half2 h1 = __hsub2(*reinterpret_cast<const __half2*>(&b1), off);
+                    const __half2 v0 = __hsub2(*reinterpret_cast<const __half2*>(&b0), off);
+                    const __half2 v1 = __hsub2(*reinterpret_cast<const __half2*>(&b1), off);
                     float c[4] = {acc[4 * w + e][0], acc[4 * w + e][1], dummy[0], dummy[1]};
-                    mma_f16(c, pa0, pa2, *reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1));
+                    mma_f16(c, pa0, pa2, *reinterpret_cast<const uint32_t*>(&v0), *reinterpret_cast<const uint32_t*>(&v1));
                     acc[4 * w + e][0] = c[0]; acc[4 * w + e][1] = c[1];
                     dummy[0] = c[2]; dummy[1] = c[3];
                 }
             }
+            if (!counts_z) z_part = 0.f;   // the row sum of a key step is counted by one of its warps
         }
-        // the next tile writes the other score buffers; the sync at its top orders the reuse of the stage
     }
 
-    // ---- partial result of this split: sum over the warps (key steps), then (m, z, O~) to the workspace ----
-    __syncthreads();   // every thread is done with the ring: reuse it for the reduction over the warps
-    float (*red)[R][D] = reinterpret_cast<float (*)[R][D]>(ring);
+    // ---- merge of the eight warps, then (m, z, O~) of this split to the workspace --------------------
+    __syncthreads();   // every warp is out of the ring (all copies it waited for have landed)
+    if (*reinterpret_cast<volatile int*>(&abort_flag)) {
+        if (tid == 0 && atomicCAS(&prm.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
+            prm.status[1] = 16; prm.status[2] = t0; prm.status[3] = 0;
+        }
+        return;
+    }
+    float (*red)[R][D + 2] = reinterpret_cast<float (*)[R][D + 2]>(ring);   // per warp and row: O~[D], m, z
     {
         const int nb0 = (warp % NSPLIT) * NBLK;
         if constexpr (NSPLIT > 1) {
@@ -366,6 +375,9 @@ decode_kernel(const DecodeParams prm) {
             for (int idx = lane; idx < R * D; idx += 32) red[warp][idx / D][idx % D] = 0.f;
             __syncwarp();
         }
+        float z = z_part;
+        z += __shfl_xor_sync(0xffffffffu, z, 1);
+        z += __shfl_xor_sync(0xffffffffu, z, 2);
         if (g < R) {
 #pragma unroll
             for (int nb = 0; nb < NBLK; ++nb) {
@@ -373,21 +385,29 @@ decode_kernel(const DecodeParams prm) {
                 red[warp][g][BPG * (2 * t) + nb0 + nb] = acc[nb][0];
                 red[warp][g][BPG * (2 * t + 1) + nb0 + nb] = acc[nb][1];
             }
+            if (t == 0) { red[warp][g][D] = m_run; red[warp][g][D + 1] = z; }
         }
     }
     __syncthreads();
-    for (int idx = tid; idx < R * D; idx += kThreads) {
+    for (int idx = tid; idx < R * D; idx += kDecodeThreads) {
         const int r = idx / D, e = idx - r * D;
-        float o = 0.f;
+        float m = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) o += red[w][r][e];
+        for (int w = 0; w < kConsumerWarps; ++w) m = fmaxf(m, red[w][r][D]);
+        float o = 0.f, z = 0.f;
+        if (m > -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const float mw = red[w][r][D];
+                if (mw == -INFINITY) continue;
+                const float wgt = exp2f(mw - m);
+                o += red[w][r][e] * wgt;
+                z += red[w][r][D + 1] * wgt;
+            }
+        }
         const int64_t row = (static_cast<int64_t>(b) * prm.Hq + hk * R + r) * prm.n_splits + split;
         prm.o_part[row * D + e] = o;
-    }
-    if (warp < R && lane == 0) {
-        const int64_t row = (static_cast<int64_t>(b) * prm.Hq + hk * R + warp) * prm.n_splits + split;
-        prm.m_part[row] = m_run;
-        prm.z_part[row] = z_run;
+        if (e == 0) { prm.m_part[row] = m; prm.z_part[row] = z; }
     }
 }
 
@@ -423,7 +443,7 @@ int launch_cfg(const DecodeParams& prm, __half* out, float* lse, cudaStream_t st
     if (e != cudaSuccess) return static_cast<int>(e);
     e = cudaMemsetAsync(prm.status, 0, 16, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
-    decode_kernel<D, R, T><<<grid, kThreads, kRing, stream>>>(prm);
+    decode_kernel<D, R, T><<<grid, kDecodeThreads, kRing, stream>>>(prm);
     g_launch_count.fetch_add(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return static_cast<int>(e);
@@ -531,9 +551,9 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     __half* out = static_cast<__half*>(out_f16);
     // keys are streamed and processed one routing tile at a time (64-key chunks with a deeper ring
     // were slower: the per-chunk barriers cost more than the extra bytes in flight gain)
-    if (p->head_dim == 128 && p->tile_n == 128) return launch_r<128, 128>(R, prm, out, lse, s);
+    if (p->head_dim == 128 && p->tile_n == 128) return launch_r<128, kChunk>(R, prm, out, lse, s);
     if (p->head_dim == 128 && p->tile_n == 64) return launch_r<128, 64>(R, prm, out, lse, s);
-    if (p->head_dim == 64 && p->tile_n == 128) return launch_r<64, 128>(R, prm, out, lse, s);
+    if (p->head_dim == 64 && p->tile_n == 128) return launch_r<64, kChunk>(R, prm, out, lse, s);
     if (p->head_dim == 64 && p->tile_n == 64) return launch_r<64, 64>(R, prm, out, lse, s);
     return TILEMIX_ERR_UNSUPPORTED;
 }
