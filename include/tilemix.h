@@ -235,7 +235,8 @@ int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varle
  * scale is folded into the probability before the PV sum (FP32 accumulation), O is written as FP16.
  * Only the K copy a group is routed to is read, so the bytes per cached token are 2*d (INT8 route)
  * or 3*d (FP16 route).  The keys are split over n_splits CTAs per (b, h_k); every CTA serves the
- * H_q/H_k query heads of its KV head; a second kernel merges the partial results.
+ * H_q/H_k query heads of its KV head (their rows fill a warp-level tensor-core tile); a second
+ * kernel merges the partial results.
  * Supported: head_dim 64 or 128, tile_n 64 or 128, H_q/H_k in {1, 2, 4, 8}. */
 typedef struct tilemix_decode {
     int32_t batch, heads_q, heads_kv, head_dim;
