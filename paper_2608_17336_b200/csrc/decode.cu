@@ -2,9 +2,9 @@
 // token per sequence, keys split over CTAs, the H_q/H_k query heads of a KV head served together.
 // HBM-bound: a cached token costs d bytes of K8 (or 2d of FP16 K on the FP16 route) plus d bytes of
 // V8, each read once: the tiles are contiguous in the cache and are streamed into a shared-memory ring
-// by untiled bulk copies, a tile ahead of their use.  All arithmetic is on the CUDA cores (dp4a for the
-// INT8 route), because with at most 8 query rows per KV head there is no tile for the tensor cores to
-// work on.
+// by untiled bulk copies, a tile ahead of their use.  The H_q/H_k query rows of a KV head are the rows of
+// a 16-row warp-level tensor-core operand (the 64-row minimum of tcgen05 has no use for 1..8 rows); on
+// the CUDA cores alone the step is instruction-bound at about a third of the HBM rate.
 #include <cuda_fp16.h>
 #include <math.h>
 
@@ -15,7 +15,6 @@ namespace tilemix {
 
 namespace {
 
-constexpr int kThreads = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -39,25 +38,8 @@ struct DecodeParams {
     int* status;     // 4 ints at the start of the workspace (same record as the attention kernel's)
 };
 
-__device__ __forceinline__ float round_to_half(float x) { return __half2float(__float2half_rn(x)); }
-
-// 4 signed bytes of `w` -> 4 floats, without the conversion unit: byte b of (w ^ 0x80808080) placed in
-// the low mantissa byte of 2^23 gives the float 2^23 + (x + 128); subtracting 2^23 + 128 is exact.
-__device__ __forceinline__ void bytes_to_floats(uint32_t w, float2 (&f)[2]) {
-    const uint32_t u = w ^ 0x80808080u;
-    const float2 bias = make_float2(-8388736.f, -8388736.f);
-    f[0] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(u, 0x4B000000u, 0x7650)),
-                                  __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7651))), bias);
-    f[1] = __fadd2_rn(make_float2(__uint_as_float(__byte_perm(u, 0x4B000000u, 0x7652)),
-                                  __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653))), bias);
-}
-
-#ifndef TILEMIX_DECODE_STAGES
-#define TILEMIX_DECODE_STAGES 2
-#define TILEMIX_DECODE_CHUNK 128
-#endif
-constexpr int kStages = TILEMIX_DECODE_STAGES;   // ring of key/value tiles in shared memory
-constexpr int kChunk = TILEMIX_DECODE_CHUNK;     // keys per kernel tile when tile_n allows it
+constexpr int kStages = 2;    // ring of key/value tiles in shared memory
+constexpr int kChunk = 128;   // keys per kernel tile when tile_n allows it (64-key tiles with deeper rings were slower)
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 
 template <int D, int T>
