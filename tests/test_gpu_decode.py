@@ -98,3 +98,33 @@ def test_decode_keys_beyond_cache_len_are_not_read():
     v2[:, :, 256:] = -7.0
     b_, _ = _gpu(q, k2, v2, route, lens, 128, 1)
     assert torch.equal(a["out"].view(torch.int16), b_["out"].view(torch.int16))
+
+
+def test_decode_zero_query_and_zero_blocks():
+    """A zero query row (delta_q = 0) and an all-zero key block (delta_K = 0): every INT8 score is 0, the
+    probabilities are uniform over the cached keys, no division by zero anywhere."""
+    q, k, v, route, lens = _case(2, 4, 2, 384, 128, 128, 1, seed=27, lens=[384, 200], f8=1.0)
+    q[0, 1] = 0
+    k[1, :, 128:256] = 0
+    _check(q, k, v, route, lens, 128, 1)
+    mixed = route.copy(); mixed[..., 1] = 0
+    _check(q, k, v, mixed, lens, 128, 1)
+
+
+def test_decode_large_magnitudes():
+    """Keys and values near the top of the FP16 range in a few channels, large score spread."""
+    q, k, v, route, lens = _case(1, 8, 2, 640, 128, 128, 1, seed=28, lens=[601])
+    k[:, :, :, 5] *= 40.0
+    q[:, :, 5] *= 6.0
+    v[:, :, 100:130, 7] = 30000.0
+    _check(q, k, v, route, lens, 128, 1)
+
+
+@pytest.mark.parametrize("seed", [31, 32, 33])
+def test_decode_random_shapes(seed):
+    rng = np.random.default_rng(seed)
+    d = int(rng.choice([64, 128])); tile = int(rng.choice([64, 128])); rep = int(rng.choice([1, 2, 4, 8]))
+    Hk = int(rng.integers(1, 4)); B = int(rng.integers(1, 5)); L = int(rng.integers(1, 1200)); G = int(rng.integers(1, 4))
+    lens = rng.integers(0, L + 1, B).tolist()
+    q, k, v, route, lens = _case(B, Hk * rep, Hk, L, d, tile, G, seed=seed, lens=lens, f8=float(rng.random()))
+    _check(q, k, v, route, lens, tile, G, n_splits=int(rng.integers(0, 6)))

@@ -130,3 +130,18 @@ def test_varlen_max_seqlen_fixes_mask_width():
     assert b["words"].shape[-1] == 2
     assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
     assert torch.equal(a["counts"], b["counts"])
+
+
+@pytest.mark.parametrize("seed", [41, 42, 43])
+def test_varlen_random_batches(seed):
+    rng = np.random.default_rng(seed)
+    big = bool(rng.integers(0, 2))
+    d = tile = 128 if big else 64
+    n = int(rng.integers(1, 7))
+    lens = rng.integers(0, 700, n).tolist()
+    if sum(lens) == 0:
+        lens[0] = 5
+    Hk = int(rng.integers(1, 3)); rep = int(rng.choice([1, 2]))
+    cu = np.cumsum([0] + lens).tolist()
+    _check_batch(cu, Hk * rep, Hk, d, tile, int(rng.integers(1, 4)), seed=seed, f8=float(rng.random()),
+                 pin=bool(rng.integers(0, 2)))
