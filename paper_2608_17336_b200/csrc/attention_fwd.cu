@@ -34,6 +34,7 @@ constexpr int kMmaWarp = 9;
 constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
 constexpr int kRegsSoftmax = 216, kRegsOther = 72;   // setmaxnreg split: 2*128*216 + 128*72 = 64512 of the 65536 registers
 constexpr int kRing = 8;
+constexpr int kBundles = 4;        // operand bundles in flight at most (each has a "landed" and a "consumed" barrier)
 constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
 constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
 constexpr uint64_t kTimeoutNs = 2000000000ull;
@@ -224,8 +225,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // ---- shared memory ------------------------------------------------------------------
     const uint32_t bar0 = sbase + C::kOffBars;
     auto bar_q = [&](int t) { return bar0 + 8u * t; };
-    auto bar_full = [&](int s) { return bar0 + 8u * (2 + s); };
-    auto bar_empty = [&](int s) { return bar0 + 8u * (2 + kRing + s); };
+    // Operands travel in bundles: bundle 0 = the K copies of key tile 0, bundle j + 1 = V_j and the K copies
+    // of key tile j + 1 -- exactly what an MMA issuer needs for its iteration j.  One "landed" barrier and
+    // one "consumed" barrier per bundle (kBundles of each, used round robin), whatever the number of
+    // chunks, so an issuer pays one wait and one commit per key tile.
+    auto bar_full = [&](int i) { return bar0 + 8u * (2 + i); };            // bundle i % kBundles landed
+    auto bar_empty = [&](int i) { return bar0 + 8u * (2 + kRing + i); };   // ... consumed by every issuer
     // per query tile t and half h of the score tile: "S half ready", "P half ready"; per tile: "PV retired"
     auto bar_s = [&](int t, int h) { return bar0 + 8u * (2 + 2 * kRing + 2 * t + h); };
     auto bar_p = [&](int t, int h) { return bar0 + 8u * (6 + 2 * kRing + 2 * t + h); };
@@ -239,9 +244,9 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar_q(0), 1);
         ptx::mbar_init(bar_q(1), 1);
-        for (int s = 0; s < kRing; ++s) {
-            ptx::mbar_init(bar_full(s), 1);
-            ptx::mbar_init(bar_empty(s), hasB ? 2 : 1);   // one arrival per MMA issuer
+        for (int i = 0; i < kBundles; ++i) {
+            ptx::mbar_init(bar_full(i), 1);
+            ptx::mbar_init(bar_empty(i), hasB ? 2 : 1);   // one arrival per MMA issuer
         }
         for (int t = 0; t < 2; ++t) {
             for (int h = 0; h < 2; ++h) {
@@ -311,39 +316,66 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (prm.has_int8)
                     ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
             }
-            // One ring item = the chunks of one operand tile.  Its data arrives on the "full" barrier
-            // of its first chunk; every chunk is handed back on its own "empty" barrier (items of
-            // different sizes reuse the chunks in different groupings).
+            // Chunks are taken from the ring in the order K16_j?, K8_j?, V_j (j = 0, 1, ...), the same
+            // order in which the issuers count them.  A chunk may be refilled once the bundle that used it
+            // last has been consumed; `last_user` remembers that bundle per chunk.
             Ring ring;
-            ring.phases = 0xffu;   // first wait on every "empty" barrier passes immediately
-            uint32_t issued = 0u, full_phase = 0u, last_parity = 0u;   // per-slot bits
             bool ok = true;
-            auto fill = [&](uint32_t s, int n_chunks, const CUtensorMap* tm, uint32_t bytes, int row) {
-                for (int c = 0; c < n_chunks && ok; ++c) {
-                    if (!wait_bar(cx, bar_empty(s + c), ring.phase(s + c), kRoleProducer, (row - tok0) / T, kBarRingEmpty)) ok = false;
-                    ring.flip(s + c);
+            int consumed = 0;                       // bundles 0 .. consumed-1 are known to be consumed
+            int last_user[kRing];
+            for (int s = 0; s < kRing; ++s) last_user[s] = -1;
+            auto wait_consumed = [&](int bundle, int j) {   // until `bundle` has been consumed
+                while (ok && consumed <= bundle) {
+                    if (!wait_bar(cx, bar_empty(consumed % kBundles), (consumed / kBundles) & 1, kRoleProducer, j, kBarRingEmpty)) ok = false;
+                    ++consumed;
                 }
-                if (!ok) return;
-                ptx::mbar_arrive_expect_tx(bar_full(s), bytes);
-                for (int c = 0; c < n_chunks; ++c)
-                    ptx::tma_load_4d(sbase + C::kOffRing + (s + c) * C::kChunk, tm, bar_full(s), c * 64, row, hk, b);
-                last_parity = (last_parity & ~(1u << s)) | (full_phase & (1u << s));
-                full_phase ^= 1u << s;
-                issued |= 1u << s;
             };
-            for (int j = 0; j < nkv && ok; ++j) {
-                const uint32_t e = sched(j);
-                if (e & 4u) fill(ring.take(C::kHalves), C::kHalves, &tm_k16, C::kHalves * C::kChunk, tok0 + j * T);
-                if (e & 8u) fill(ring.take(1), 1, &tm_k8, C::kK8Bytes, tok0 + j * T);
-                fill(ring.take(C::kHalves), C::kHalves, &tm_v16, C::kHalves * C::kChunk, tok0 + j * T);
+            int armed = 0;                          // bundles whose copies have been issued
+            for (int n = 0; n <= nkv && ok; ++n) {
+                // bundle n: V of key tile n - 1 (n >= 1) and the K copies of key tile n (n < nkv)
+                const uint32_t e = n < nkv ? sched(n) : 0u;
+                const bool has_v = n >= 1;
+                uint32_t s16 = 0, s8 = 0, sv = 0, bytes = 0;
+                // chunk order inside the sequence: ..., V_{n-1}, K16_n, K8_n, V_n, ...
+                if (has_v) { sv = ring.take(C::kHalves); bytes += C::kHalves * C::kChunk; }
+                if (e & 4u) { s16 = ring.take(C::kHalves); bytes += C::kHalves * C::kChunk; }
+                if (e & 8u) { s8 = ring.take(1); bytes += C::kK8Bytes; }
+                if (bytes == 0u) break;             // nothing after the last V
+                if (n >= kBundles) wait_consumed(n - kBundles, n);     // its barriers are free again
+                // the barrier is armed for the whole bundle first; every operand is then copied as soon as
+                // its own chunks are free, so a V tile does not wait for the room of the K tile behind it
+                const uint32_t bar = bar_full(n % kBundles);
+                ptx::mbar_arrive_expect_tx(bar, bytes);
+                armed = n + 1;
+                auto claim = [&](uint32_t slot, int chunks) {
+                    for (int c = 0; c < chunks; ++c) {
+                        if (last_user[slot + c] >= 0) wait_consumed(last_user[slot + c], n);
+                        last_user[slot + c] = n;
+                    }
+                };
+                if (has_v) {
+                    claim(sv, C::kHalves);
+                    if (!ok) break;
+                    for (int c = 0; c < C::kHalves; ++c)
+                        ptx::tma_load_4d(sbase + C::kOffRing + (sv + c) * C::kChunk, &tm_v16, bar, c * 64, tok0 + (n - 1) * T, hk, b);
+                }
+                if (e & 4u) {
+                    claim(s16, C::kHalves);
+                    if (!ok) break;
+                    for (int c = 0; c < C::kHalves; ++c)
+                        ptx::tma_load_4d(sbase + C::kOffRing + (s16 + c) * C::kChunk, &tm_k16, bar, c * 64, tok0 + n * T, hk, b);
+                }
+                if (e & 8u) {
+                    claim(s8, 1);
+                    if (!ok) break;
+                    ptx::tma_load_4d(sbase + C::kOffRing + s8 * C::kChunk, &tm_k8, bar, 0, tok0 + n * T, hk, b);
+                }
             }
             if (!ok || *cx.abort_flag) {
                 // let copies that are still in flight land before the CTA's memory is released
-                for (uint32_t s = 0; s < kRing; ++s) {
-                    if (!(issued >> s & 1u)) continue;
+                for (int n = armed > kBundles ? armed - kBundles : 0; n < armed; ++n)
                     for (int it = 0; it < (1 << 20); ++it)
-                        if (ptx::mbar_try_wait(bar_full(s), (last_parity >> s) & 1u)) break;
-                }
+                        if (ptx::mbar_try_wait(bar_full(n % kBundles), (n / kBundles) & 1)) break;
             }
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
@@ -360,13 +392,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             constexpr uint32_t kIdescPV = ptx::instr_desc(1, 0, 0, 1, C::kM, D);
             Ring ring;
             bool ok = true;
-            // Wait until chunk s holds its data.  An issuer waits for EVERY item, also those whose data
-            // it does not read: its arrival on the item's "empty" barrier must not run a ring cycle
-            // ahead of the other issuer's, or two arrivals of one issuer would release the chunk.
-            auto acquire = [&](uint32_t s, int j) {
+            // Wait until bundle n has landed.  An issuer waits for EVERY bundle, also one whose data it
+            // does not read: its arrival on the bundle's "consumed" barrier must not run a round of the
+            // barriers ahead of the other issuer's, or two arrivals of one issuer would release it.
+            auto acquire = [&](int n) {
                 if (!ok) return;
-                if (!wait_bar(cx, bar_full(s), ring.phase(s), kRoleMma, j, kBarRingFull)) ok = false;
-                ring.flip(s);
+                if (!wait_bar(cx, bar_full(n % kBundles), (n / kBundles) & 1, kRoleMma, n, kBarRingFull)) ok = false;
             };
             // Descriptor words that do not change: the high words, and the low words of the
             // resident Q operands.  One K step advances a K-major operand by 32 bytes inside its
@@ -419,16 +450,16 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             // slots of the K operands of the tile whose QK^T is issued next
             uint32_t e_next = sched(0), k16 = 0, k8 = 0;
             uint32_t r_next = (e_next >> t) & 1u;          // route of this tile at the next key tile
-            if (e_next & 4u) { k16 = ring.take(C::kHalves); acquire(k16, 0); }
-            if (e_next & 8u) { k8 = ring.take(1); acquire(k8, 0); }
+            if (e_next & 4u) k16 = ring.take(C::kHalves);
+            if (e_next & 8u) k8 = ring.take(1);
+            acquire(0);
             if (ok) {
                 ptx::tc_fence_after_sync();
                 for (int h = 0; h < 2; ++h) {
                     issue_qk(t, h, r_next, k16, k8);
                     ptx::mma_commit(bar_s(t, h));
                 }
-                if (e_next & 4u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
-                if (e_next & 8u) ptx::mma_commit(bar_empty(k8));
+                ptx::mma_commit(bar_empty(0));
             }
             for (int j = 0; j < nkv && ok; ++j) {
                 const bool mine = j <= m_t;            // tile A has no work at the last key tile of tile B
@@ -438,10 +469,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 r_next = (e_next >> t) & 1u;
                 if (e_next & 4u) k16 = ring.take(C::kHalves);
                 if (e_next & 8u) k8 = ring.take(1);
-                // operands of this iteration: wait for them now, off the P -> PV critical path
-                acquire(sv, j);
-                if (e_next & 4u) acquire(k16, j + 1);
-                if (e_next & 8u) acquire(k8, j + 1);
+                // operands of this iteration (bundle j + 1): wait for them now, off the P -> PV critical path
+                acquire(j + 1);
                 if (!ok) break;
                 // Half steps: as soon as P of a half has arrived its PV is issued, and right behind it the
                 // QK^T of the NEXT key tile into the same half of S_t -- the softmax group is meanwhile
@@ -469,9 +498,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     }
                 }
                 if (!ok) break;
-                for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(sv + c));
-                if (e_next & 4u) for (int c = 0; c < C::kHalves; ++c) ptx::mma_commit(bar_empty(k16 + c));
-                if (e_next & 8u) ptx::mma_commit(bar_empty(k8));
+                ptx::mma_commit(bar_empty((j + 1) % kBundles));
             }
             // every MMA issued by this thread has retired before TMEM / shared memory go away
             ptx::mma_commit(bar_drain);
