@@ -108,6 +108,9 @@ decode_kernel(const DecodeParams prm) {
     __shared__ float dq_s[R];
     __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
     __shared__ int abort_flag;
+    // route bit (sign) and the two block scales of the first kMetaTiles tiles of this split, staged once
+    constexpr int kMetaTiles = 256;
+    __shared__ float2 meta[kMetaTiles];   // x = delta_K (negative zero / negated: FP16 route), y = delta_V
 
     const uint32_t ring_u32 = ptx::smem_u32(ring);
     if (tid == 0) {
@@ -178,7 +181,12 @@ decode_kernel(const DecodeParams prm) {
         }
         return true;
     };
-    __syncthreads();   // barriers initialised, query rows staged
+    for (int i = tid; i < kMetaTiles && t0 + i < t1; i += kDecodeThreads) {
+        const int tile = t0 + i;
+        // delta_K >= 0; the FP16 route is marked by a negative x (its delta_K is not used)
+        meta[i] = make_float2(route_of(tile) ? dk[tile / per_blk] : -1.f, dv[tile / per_blk]);
+    }
+    __syncthreads();   // barriers initialised, query rows and tile metadata staged
 
     // per-warp flash-decoding state: rows g (< R) of this warp's keys
     float m_run = -INFINITY, z_part = 0.f;          // z_part: this lane's share of the row sum
@@ -222,9 +230,19 @@ decode_kernel(const DecodeParams prm) {
         for (int tile = t0; tile < t1; ++tile) {
             const int it = tile - t0, stage = it % kStages;
             if (producer && tile + kStages - 1 < t1) produce(tile + kStages - 1);   // keeps the ring full
-            const bool int8 = route_of(tile);
-            // ahead of the wait (fetching them a tile ahead instead costs registers and was slower)
-            const float dkt = int8 ? dk[tile / per_blk] : 0.f, dvt = dv[tile / per_blk];
+            // route bit and block scales: from shared memory (global loads for tiles beyond the staged ones)
+            bool int8;
+            float dkt, dvt;
+            if (it < kMetaTiles) {
+                const float2 mt = meta[it];
+                int8 = mt.x >= 0.f;
+                dkt = mt.x;
+                dvt = mt.y;
+            } else {
+                int8 = route_of(tile);
+                dkt = int8 ? dk[tile / per_blk] : 0.f;
+                dvt = dv[tile / per_blk];
+            }
             if (!wait_ring(&full_bar[stage], (it / kStages) & 1)) break;
             const uint8_t* kst = ring + stage * St::kBytes;
             const uint8_t* vst = kst + St::kK;
