@@ -121,6 +121,22 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
                           void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg,
                           void* stream);
 
+/* Chunked prefill: the queries are the LAST p->seqlen tokens of a context of kv_len tokens whose keys
+ * and values are all present (earlier chunks, a prefix cache); query i attends to keys
+ * 0 .. kv_len - p->seqlen + i.  The result equals the corresponding rows of tilemix_attention_fwd over
+ * the whole context, bit for bit.  kv_len - p->seqlen must be a multiple of the tile (so that query
+ * tiles, quantisation blocks and mask rows line up with the context's).
+ *   q_f16, q_i8, out_f16   [B,Hq,seqlen,d];  q_scale [B,Hq,ceil(seqlen/tile)];  lse [B,Hq,seqlen]
+ *   k_f16, v_f16, k_i8     [B,Hk,kv_len,d] (dense strides are taken with kv_len);  k_scale [B,Hk,ceil(kv_len/tile)]
+ *   mask_words             the words of the WHOLE context, uint32 [nb,Hk,ceil(kv_len/tile),W(kv_len)], as
+ *                          tilemix_pack_routing_mask writes them for seqlen = kv_len; the chunk reads its rows
+ * Everything else as for tilemix_attention_fwd (the workspace needs 4096 bytes). */
+int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, const void* q_f16,
+                                const void* k_f16, const void* v_f16, const int8_t* q_i8,
+                                const int8_t* k_i8, const float* q_scale, const float* k_scale,
+                                const uint32_t* mask_words, void* out_f16, float* lse, void* workspace,
+                                size_t workspace_bytes, const tilemix_debug_t* dbg, void* stream);
+
 /* Same computation as tilemix_attention_fwd for callers that cannot hand it a workspace because
  * they cannot allocate device memory at all: a process whose whole GPU memory was claimed at
  * start-up by another allocator or memory pool (any later cudaMalloc fails), or a code path that

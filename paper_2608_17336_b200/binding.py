@@ -23,7 +23,7 @@ EXPORTS = (
     "tilemix_read_status", "tilemix_status_string", "tilemix_launch_count",
     "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
     "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
-    "tilemix_decode_workspace_size", "tilemix_decode_int8kv",
+    "tilemix_decode_workspace_size", "tilemix_decode_int8kv", "tilemix_attention_fwd_chunk",
 )
 
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.tilemix_pack_routing_mask.argtypes = [pp, vp, u32, vp, vp, vp]
         L.tilemix_attention_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t,
                                             ctypes.POINTER(DebugStruct), vp]
+        L.tilemix_attention_fwd_chunk.argtypes = [pp, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                  ctypes.c_size_t, ctypes.POINTER(DebugStruct), vp]
         L.tilemix_attention_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                                     ctypes.POINTER(DebugStruct), ctypes.POINTER(vp), vp]
         L.tilemix_prefill_host.argtypes = [pp, vp, vp, vp, vp, u32, vp, vp, ctypes.c_size_t, vp]
@@ -386,3 +388,23 @@ def tilemix_decode_int8kv(p: DecodeStruct, q, k16, k8, k_scale, v8, v_scale, wor
                                      _ptr(qs), _ptr(workspace), workspace.numel(), _stream())
     _check(rc, "tilemix_decode_int8kv")
     return {"out": out, "lse": lse, "q8": q8, "q_scale": qs, "workspace": workspace}
+
+
+# ------------------------------------------------------------------ chunked prefill
+
+def tilemix_attention_fwd_chunk(p: ProblemStruct, kv_len: int, q, k, v, q8, k8, q_scale, k_scale, words, out=None,
+                                want_lse=False, workspace=None):
+    """The last p.seqlen queries of a kv_len-token context: q [B,Hq,seqlen,d], k/v [B,Hk,kv_len,d], words
+    those of the whole context.  Returns a dict like tilemix_attention_fwd."""
+    dev = q.device
+    if out is None:
+        out = torch.empty((p.batch, p.heads_q, p.seqlen, p.head_dim), dtype=torch.float16, device=dev)
+    lse = torch.empty((p.batch, p.heads_q, p.seqlen), dtype=torch.float32, device=dev) if want_lse else None
+    if workspace is None:
+        workspace = torch.empty(4096, dtype=torch.uint8, device=dev)
+    pp = _with_strides(p, q=q, k=k, v=v, o=out)
+    rc = lib().tilemix_attention_fwd_chunk(ctypes.byref(pp), kv_len, _ptr(q), _ptr(k), _ptr(v), _ptr(q8), _ptr(k8),
+                                           _ptr(q_scale), _ptr(k_scale), _ptr(words), _ptr(out), _ptr(lse),
+                                           _ptr(workspace), workspace.numel(), None, _stream())
+    _check(rc, "tilemix_attention_fwd_chunk")
+    return {"out": out, "lse": lse, "workspace": workspace}

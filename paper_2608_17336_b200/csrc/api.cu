@@ -65,6 +65,7 @@ int resolve(const tilemix_problem_t* p, Geometry* g) {
     g->T_n = static_cast<int>(ceil_div(g->L, g->tile_n));
     g->T_mask = static_cast<int>(ceil_div(g->L, static_cast<int64_t>(g->G) * g->tile_n));
     g->W = static_cast<int>(ceil_div(g->T_mask, 32));
+    g->Lk = g->L; g->kv_off = 0; g->mask_T_m = g->T_m; g->ks_blocks = static_cast<int>(ceil_div(g->L, g->blk_k));
     g->scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(g->d));
     g->flags = p->flags;
     int rc;
@@ -130,6 +131,47 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
         (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
         return TILEMIX_ERR_ALIGN;
     if (workspace_bytes < tilemix_workspace_size(p)) return TILEMIX_ERR_WORKSPACE;
+    if ((rc = check_device())) return rc;
+    return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
+                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+}
+
+int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, const void* q_f16, const void* k_f16,
+                                const void* v_f16, const int8_t* q_i8, const int8_t* k_i8, const float* q_scale,
+                                const float* k_scale, const uint32_t* mask_words, void* out_f16, float* lse,
+                                void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg, void* stream) {
+    if (p == nullptr) return TILEMIX_ERR_NULL;
+    if (kv_len < p->seqlen || p->tile_m <= 0 || p->tile_m != p->tile_n || (kv_len - p->seqlen) % p->tile_m != 0)
+        return TILEMIX_ERR_SHAPE;
+    // K and V are kv_len tokens long: dense strides are theirs, not the chunk's
+    tilemix_problem_t q = *p;
+    if (all_zero(q.k_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.k_stride);
+    if (all_zero(q.v_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.v_stride);
+    Geometry g;
+    int rc = resolve(&q, &g);
+    if (rc) return rc;
+    g.Lk = kv_len;
+    g.kv_off = (kv_len - g.L) / g.tile_m;
+    g.T_n = static_cast<int>(ceil_div(kv_len, g.tile_n));
+    g.mask_T_m = g.T_n;                      // the mask words of the whole context
+    g.ks_blocks = static_cast<int>(ceil_div(kv_len, g.blk_k));
+    g.T_mask = static_cast<int>(ceil_div(kv_len, static_cast<int64_t>(g.G) * g.tile_n));
+    g.W = static_cast<int>(ceil_div(g.T_mask, 32));
+    if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
+    const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
+    if (!force16 && !(q_i8 && k_i8 && q_scale && k_scale && mask_words)) return TILEMIX_ERR_NULL;
+    if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
+    if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
+    const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
+                          (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
+    if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
+    if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
+        !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
+        (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
+        return TILEMIX_ERR_ALIGN;
+    if (workspace_bytes < 4096) return TILEMIX_ERR_WORKSPACE;
     if ((rc = check_device())) return rc;
     return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
                             k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));

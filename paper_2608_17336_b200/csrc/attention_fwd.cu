@@ -86,6 +86,7 @@ struct Cfg {
 
 struct Params {
     int B, Hq, Hk, L, G, T_m, W, nb;
+    int kv_off, mask_T_m, ks_blocks;   // chunked prefill: see Geometry (0, T_m, T_m for a plain prefill)
     int has_int8;                 // INT8 operands present
     float scale_log2;             // softmax scale * log2(e)
     const float* q_scale;         // [B,Hq,T_m]; variable-length batch: [sum T_m, Hq]
@@ -197,7 +198,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // b: batch coordinate of the tensor maps; seq: sequence index (== b for a dense batch);
     // tok0 / len: first token and length of the sequence; row0: its first row among the mask rows
     // and scale blocks; m, n below count tiles inside the sequence.
-    int b, hq, pr, seq, tok0 = 0, len = prm.L, row0 = 0, n_rows = prm.T_m;
+    int b, hq, pr, seq, tok0 = 0, len = prm.L, row0 = VL ? 0 : prm.kv_off, n_rows = prm.T_m;
     if constexpr (!VL) {
         const int n_pairs = (prm.T_m + 1) >> 1;
         const int bh = blockIdx.x / n_pairs;
@@ -218,9 +219,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     }
     constexpr bool varlen = VL;
     const int hk = hq / (prm.Hq / prm.Hk);
+    // m: query-tile rows of this CTA (inside the sequence / the chunk); k: the key tile on their diagonal
+    // (m + the chunk's offset in the context)
+    const int kv_off = VL ? 0 : prm.kv_off;
     const int mA = 2 * pr, mB = 2 * pr + 1;
     const bool hasB = mB < n_rows;
-    const int nkv = (hasB ? mB : mA) + 1;
+    const int kA = mA + kv_off, kB = mB + kv_off;
+    const int nkv = (hasB ? kB : kA) + 1;
 
     // ---- shared memory ------------------------------------------------------------------
     const uint32_t bar0 = sbase + C::kOffBars;
@@ -272,11 +277,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if (prm.words != nullptr) {
                 const int g = j / prm.G;
                 const int nbi = (prm.nb == 1) ? 0 : b;
-                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.T_m + row0 + mA) * prm.W;
+                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.mask_T_m + row0 + mA) * prm.W;
                 e |= (rowA[g >> 5] >> (g & 31)) & 1u;
                 if (hasB) e |= ((rowA[prm.W + (g >> 5)] >> (g & 31)) & 1u) << 1;
             }
-            const bool useA = j <= mA;
+            const bool useA = j <= kA;
             if ((useA && !(e & 1u)) || (hasB && !(e & 2u))) e |= 4u;
             if ((useA && (e & 1u)) || (hasB && (e & 2u))) e |= 8u;
             packed |= e << (4 * jj);
@@ -385,7 +390,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         ptx::setmaxnreg_dec<kRegsOther>();
         if (lane == 0) {
             const int t = warp - kMmaWarp;
-            const int m_t = t ? mB : mA;
+            const int m_t = t ? kB : kA;       // last key tile of this issuer's query tile
             constexpr int TH = C::kTH;
             constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, C::kM, TH);
             constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, C::kM, TH);
@@ -508,7 +513,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         // ================================================================ softmax groups
         ptx::setmaxnreg_inc<kRegsSoftmax>();
         const int t = warp / kWarpsPerGroup;
-        const int m_t = t ? mB : mA;
+        const int m_t = t ? mB : mA;           // query-tile row
+        const int k_t = t ? kB : kA;           // its diagonal key tile
         if (t == 0 || hasB) {
             const int quarter = warp & 3;
             const int row = quarter * 32 + lane;
@@ -525,7 +531,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                                       : prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t];
             const float* dk_row = !prm.has_int8 ? nullptr
                                   : varlen ? prm.k_scale + static_cast<int64_t>(row0) * prm.Hk + hk
-                                           : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.T_m;
+                                           : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.ks_blocks;
             float m_run = -INFINITY, z = 0.f;
             float m_seen = -INFINITY;     // largest scaled score seen so far (m_run may lag it)
             bool ok = true;
@@ -538,7 +544,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             float a = prm.scale_log2;
             uint32_t int8_route = 0u;
             constexpr int TH = C::kTH;
-            const int n_steps = 2 * (m_t + 1);
+            const int n_steps = 2 * (k_t + 1);
             // One step = one half (TH key columns) of a score tile: while this group works on one half
             // of S_t, the tensor pipe runs the PV of the previous half and the QK^T of the next one
             // into the other half.  u = 2*j + h.
@@ -555,7 +561,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         a *= dq * dk_next;
                         if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                     }
-                    if (prm.has_int8 && j < m_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
+                    if (prm.has_int8 && j < k_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
                 }
                 const uint32_t t_sh = t_s + h * TH;
 #ifdef TILEMIX_PHASE_TIMERS
@@ -585,7 +591,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 // time with the next 32 already in flight from tensor memory, while its row maximum is
                 // tracked on the side; only if some row of the warp does exceed m + kTau (rare after
                 // the first tiles) the half tile is re-read and redone in the generic two-pass form.
-                const bool diag = (j == m_t);
+                const bool diag = (j == k_t);
                 bool redo = diag || j == 0 || prm.dbg_n > 0;
                 float alpha = 1.f, sum = 0.f;
                 bool grow = false;
@@ -611,7 +617,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     prefetched = false;
                     // next step: one-pass as well (not the first or the diagonal tile), and its S half ready?
                     const int jn = (u + 1) >> 1, hn = (u + 1) & 1;
-                    const bool next_fast = u + 1 < n_steps && jn != m_t;
+                    const bool next_fast = u + 1 < n_steps && jn != k_t;
                     auto late = [&]() {
                         if (next_fast && __all_sync(0xffffffffu, ptx::mbar_test_wait(bar_s(t, hn), jn & 1))) {
                             ptx::tc_fence_after_sync();
@@ -745,7 +751,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(33 + t, clock64() - loop_c0);
 #endif
             if (ok) {
-                ok = wait_bar(cx, bar_o(t), 0, role, m_t + 1, kBarO);
+                ok = wait_bar(cx, bar_o(t), 0, role, k_t + 1, kBarO);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (ok) {
@@ -837,20 +843,21 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     const bool has8 = !(g.flags & TILEMIX_FORCE_FP16) && q8 != nullptr;
     CUtensorMap tq, tk, tv, tq8, tk8;
     if ((rc = encode_map(enc, &tq, q, 2, g.d, g.L, g.Hq, g.B, g.qs, 64, C::kM, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
-    if ((rc = encode_map(enc, &tk, k, 2, g.d, g.L, g.Hk, g.B, g.ks, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
-    if ((rc = encode_map(enc, &tv, v, 2, g.d, g.L, g.Hk, g.B, g.vs, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
+    if ((rc = encode_map(enc, &tk, k, 2, g.d, g.Lk, g.Hk, g.B, g.ks, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
+    if ((rc = encode_map(enc, &tv, v, 2, g.d, g.Lk, g.Hk, g.B, g.vs, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
     if (has8) {
         const CUtensorMapSwizzle sw8 = (D == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
         const int64_t dq[3] = {static_cast<int64_t>(g.Hq) * g.L * g.d, static_cast<int64_t>(g.L) * g.d, g.d};
-        const int64_t dk[3] = {static_cast<int64_t>(g.Hk) * g.L * g.d, static_cast<int64_t>(g.L) * g.d, g.d};
+        const int64_t dk[3] = {static_cast<int64_t>(g.Hk) * g.Lk * g.d, static_cast<int64_t>(g.Lk) * g.d, g.d};
         if ((rc = encode_map(enc, &tq8, q8, 1, g.d, g.L, g.Hq, g.B, dq, D, C::kM, sw8))) return rc;
-        if ((rc = encode_map(enc, &tk8, k8, 1, g.d, g.L, g.Hk, g.B, dk, D, T, sw8))) return rc;
+        if ((rc = encode_map(enc, &tk8, k8, 1, g.d, g.Lk, g.Hk, g.B, dk, D, T, sw8))) return rc;
     } else {
         tq8 = tq;
         tk8 = tk;
     }
     Params prm{};
     prm.B = g.B; prm.Hq = g.Hq; prm.Hk = g.Hk; prm.L = g.L; prm.G = g.G; prm.T_m = g.T_m; prm.W = g.W;
+    prm.kv_off = g.kv_off; prm.mask_T_m = g.mask_T_m; prm.ks_blocks = g.ks_blocks;
     prm.nb = g.nb;
     prm.has_int8 = has8 ? 1 : 0;
     prm.scale_log2 = g.scale * kLog2e;

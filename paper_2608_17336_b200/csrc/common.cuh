@@ -23,6 +23,10 @@ struct Geometry {
     int blk_q, blk_k;
     int nb;                 // mask batch
     int T_m, T_n, T_mask, W;
+    // Chunked prefill (queries = the last L tokens of an Lk-token context): K/V length, the chunk's
+    // first tile row in the context, rows per head of the mask words, blocks per head of k_scale.
+    // For a plain prefill: Lk = L, kv_off = 0, mask_T_m = T_m, ks_blocks = T_n.
+    int Lk, kv_off, mask_T_m, ks_blocks;
     float scale;            // softmax scale (natural-log domain)
     uint32_t flags;
     int64_t qs[3], ks[3], vs[3], os[3];   // element strides (batch, head, token)

@@ -82,6 +82,7 @@ int resolve_varlen(const tilemix_problem_t* p, const tilemix_varlen_t* vl, Geome
         t->tab[base + items.size() + i] = items[i].first;
     }
     g->T_m = t->total_tiles;
+    g->mask_T_m = t->total_tiles;
     g->T_n = static_cast<int>(ceil_div(t->max_len, g->tile_n));
     g->T_mask = static_cast<int>(ceil_div(t->max_len, static_cast<int64_t>(g->G) * g->tile_n));
     g->W = static_cast<int>(ceil_div(g->T_mask, 32));
