@@ -461,6 +461,27 @@ def main():
         line["varlen"] = varlen_leg(tm, w, dev, peaks)
     if world == 1 and not args.no_decode and w.tile == 128:
         line["decode"] = decode_leg(tm, w, dev, peaks)
+    if world == 1 and not args.no_varlen and w.tile == 128 and w.batch == 1 and w.seqlen >= 8 * w.tile:
+        # chunked prefill: the last eighth of the context as a chunk against all of its keys (same tensors)
+        Lq = (w.seqlen // 8) // w.tile * w.tile
+        off = w.seqlen - Lq
+        pc = tm.problem(1, w.heads, w.heads, Lq, w.head_dim, w.tile, w.tile, w.group)
+        q8f, k8f, qsf, ksf = tm.tilemix_quantize_qk(p, qd, kd)
+        words_f, _ = tm.tilemix_pack_routing_mask(p, rd, w.pin_diagonal)
+        qc, q8c, qsc = qd[:, :, off:].contiguous(), q8f[:, :, off:].contiguous(), qsf[:, :, off // w.tile:].contiguous()
+        oc = torch.empty_like(qc)
+        for _ in range(3):
+            tm.tilemix_attention_fwd_chunk(pc, w.seqlen, qc, kd, vd, q8c, k8f, qsc, ksf, words_f, out=oc, workspace=work)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(stream)
+        for _ in range(5):
+            tm.tilemix_attention_fwd_chunk(pc, w.seqlen, qc, kd, vd, q8c, k8f, qsc, ksf, words_f, out=oc, workspace=work)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        ms = c0.elapsed_time(c1) / 5
+        fl = 4.0 * w.heads * w.head_dim * (float(Lq) * off + float(Lq) ** 2 / 2.0)
+        line["chunk"] = {"chunk_len": Lq, "context_len": w.seqlen, "attention_ms": ms,
+                         "tflops": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s"}
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
         line["cpu_baseline"] = {"value": 4.0 * w.head_dim * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": threads,
