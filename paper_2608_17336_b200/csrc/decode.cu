@@ -38,7 +38,8 @@ struct DecodeParams {
     int* status;     // 4 ints at the start of the workspace (same record as the attention kernel's)
 };
 
-constexpr int kStages = 2;    // ring of key/value tiles in shared memory
+constexpr int kStages = 2;    // ring of key/value tiles in shared memory when FP16 keys may be read ...
+constexpr int kStagesInt8 = 3;   // ... and when there is no FP16 key cache (a stage is a third smaller)
 constexpr int kChunk = 128;   // keys per kernel tile when tile_n allows it (64-key tiles with deeper rings were slower)
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 
@@ -82,7 +83,7 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a2,
 constexpr int kConsumerWarps = 8;
 constexpr int kDecodeThreads = kConsumerWarps * 32;   // 2 CTAs/SM = 4 warps per scheduler: 128 registers each
 
-template <int D, int R, int T>
+template <int D, int R, int T, bool F16K>
 __global__ void __launch_bounds__(kDecodeThreads, 2)
 decode_kernel(const DecodeParams prm) {
     using St = Stage<D, T>;
@@ -92,7 +93,7 @@ decode_kernel(const DecodeParams prm) {
     constexpr int NBLK = D / 8 / NSPLIT;          // column blocks per warp
     constexpr int BPG = D / 8;                    // bytes of a cached V row per lane group
     static_assert(KS3 <= kConsumerWarps && kConsumerWarps % KS3 == 0, "tile shape vs warps");
-    static_assert(kStages * St::kBytes >= static_cast<int>(kConsumerWarps * R * (D + 2) * sizeof(float)),
+    static_assert(kStagesInt8 * 2 * St::kV >= static_cast<int>(kConsumerWarps * R * (D + 2) * sizeof(float)),
                   "the final merge reuses the ring");
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -102,11 +103,15 @@ decode_kernel(const DecodeParams prm) {
     const int per_split = (n_tiles + prm.n_splits - 1) / prm.n_splits;
     const int t0 = split * per_split, t1 = min(n_tiles, t0 + per_split);
 
-    extern __shared__ __align__(128) uint8_t ring[];   // kStages x (K tile | V tile)
+    extern __shared__ __align__(128) uint8_t ring[];   // n_stages x (K tile | V tile)
+    // without an FP16 key cache a K slot only ever holds INT8 keys: smaller stages, one more of them
+    constexpr int n_stages = F16K ? kStages : kStagesInt8;
+    constexpr int k_slot = F16K ? St::kK : St::kV;
+    constexpr int stage_bytes = k_slot + St::kV;
     __shared__ __align__(16) uint32_t qh[R][D / 2];   // query rows, FP16 pairs (FP16 route)
     __shared__ __align__(16) uint32_t q8w[R][D / 4];  // quantised query rows, 4 bytes per word (INT8 route)
     __shared__ float dq_s[R];
-    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages];
+    __shared__ __align__(8) uint64_t full_bar[kStagesInt8], empty_bar[kStagesInt8];
     __shared__ int abort_flag;
     // route bit (sign) and the two block scales of the first kMetaTiles tiles of this split, staged once
     constexpr int kMetaTiles = 256;
@@ -114,7 +119,7 @@ decode_kernel(const DecodeParams prm) {
 
     const uint32_t ring_u32 = ptx::smem_u32(ring);
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStagesInt8; ++s) {
             ptx::mbar_init(ptx::smem_u32(&full_bar[s]), 1);
             ptx::mbar_init(ptx::smem_u32(&empty_bar[s]), kConsumerWarps);
         }
@@ -200,23 +205,23 @@ decode_kernel(const DecodeParams prm) {
     const int8_t* v8 = prm.v8 + row_base * D;
     const __half* k16 = prm.k16 != nullptr ? prm.k16 + row_base * D : nullptr;
     auto produce = [&](int tile) -> bool {
-        const int it = tile - t0, stage = it % kStages;
+        const int it = tile - t0, stage = it % n_stages;
         // the first pass over the ring finds every stage free
-        if (it >= kStages && !wait_ring(&empty_bar[stage], ((it / kStages) - 1) & 1)) return false;
+        if (it >= n_stages && !wait_ring(&empty_bar[stage], ((it / n_stages) - 1) & 1)) return false;
         const uint32_t rows = static_cast<uint32_t>(min(T, len - tile * T));   // only rows that exist
         const uint32_t bar = ptx::smem_u32(&full_bar[stage]);
-        const uint32_t dst = ring_u32 + stage * St::kBytes;
+        const uint32_t dst = ring_u32 + stage * stage_bytes;
         const bool int8 = route_of(tile);
         const uint32_t kbytes = rows * D * (int8 ? 1u : 2u);
         ptx::mbar_arrive_expect_tx(bar, kbytes + rows * D);
         if (int8) ptx::bulk_load_1d(dst, k8 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
         else ptx::bulk_load_1d(dst, k16 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
-        ptx::bulk_load_1d(dst + St::kK, v8 + static_cast<int64_t>(tile) * T * D, rows * D, bar);
+        ptx::bulk_load_1d(dst + k_slot, v8 + static_cast<int64_t>(tile) * T * D, rows * D, bar);
         return true;
     };
     const bool producer = warp == kConsumerWarps - 1 && lane == 0;
     if (producer)
-        for (int s = 0; s < kStages - 1 && t0 + s < t1; ++s) produce(t0 + s);
+        for (int s = 0; s < n_stages - 1 && t0 + s < t1; ++s) produce(t0 + s);
     {
         // ================================================================ consumers
         const int ks = warp / NSPLIT, nb0 = (warp % NSPLIT) * NBLK;   // this warp's keys and column blocks
@@ -228,8 +233,8 @@ decode_kernel(const DecodeParams prm) {
         const float dq = g < R ? dq_s[g < R ? g : 0] : 0.f;
 
         for (int tile = t0; tile < t1; ++tile) {
-            const int it = tile - t0, stage = it % kStages;
-            if (producer && tile + kStages - 1 < t1) produce(tile + kStages - 1);   // keeps the ring full
+            const int it = tile - t0, stage = it % n_stages;
+            if (producer && tile + n_stages - 1 < t1) produce(tile + n_stages - 1);   // keeps the ring full
             // route bit and block scales: from shared memory (global loads for tiles beyond the staged ones)
             bool int8;
             float dkt, dvt;
@@ -243,9 +248,9 @@ decode_kernel(const DecodeParams prm) {
                 dkt = int8 ? dk[tile / per_blk] : 0.f;
                 dvt = dv[tile / per_blk];
             }
-            if (!wait_ring(&full_bar[stage], (it / kStages) & 1)) break;
-            const uint8_t* kst = ring + stage * St::kBytes;
-            const uint8_t* vst = kst + St::kK;
+            if (!wait_ring(&full_bar[stage], (it / n_stages) & 1)) break;
+            const uint8_t* kst = ring + stage * stage_bytes;
+            const uint8_t* vst = kst + k_slot;
             // ---- (1) scores of this warp's 16 keys, rows g: s[nb][0..1] = keys 8 nb + 2t, 2t + 1 ----------
             float sc[2][2];
             if (int8) {
@@ -438,12 +443,15 @@ decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ 
 template <int D, int R, int T>
 int launch_cfg(const DecodeParams& prm, __half* out, float* lse, cudaStream_t stream) {
     const dim3 grid(prm.n_splits, prm.Hk, prm.B);
-    constexpr int kRing = kStages * Stage<D, T>::kBytes;
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, R, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRing);
+    constexpr int kRing = kStages * Stage<D, T>::kBytes;   // = kStagesInt8 stages of INT8 keys and values
+    static_assert(kRing == kStagesInt8 * 2 * Stage<D, T>::kV, "both ring shapes fill the same bytes");
+    // no FP16 key cache: the instance whose ring holds three INT8-only stages
+    auto kernel = prm.k16 != nullptr ? decode_kernel<D, R, T, true> : decode_kernel<D, R, T, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRing);
     if (e != cudaSuccess) return static_cast<int>(e);
     e = cudaMemsetAsync(prm.status, 0, 16, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
-    decode_kernel<D, R, T><<<grid, kDecodeThreads, kRing, stream>>>(prm);
+    kernel<<<grid, kDecodeThreads, kRing, stream>>>(prm);
     g_launch_count.fetch_add(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return static_cast<int>(e);
