@@ -592,7 +592,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 // tracked on the side; only if some row of the warp does exceed m + kTau (rare after
                 // the first tiles) the half tile is re-read and redone in the generic two-pass form.
                 const bool diag = (j == k_t);
-                bool redo = diag || j == 0 || prm.dbg_n > 0;
+                bool redo = diag || u == 0 || prm.dbg_n > 0;
                 float alpha = 1.f, sum = 0.f;
                 bool grow = false;
                 uint32_t p2[TH / 2];
@@ -615,7 +615,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     float mx;
                     if (!prefetched) ptx::tmem_ld32(t_sh, first);
                     prefetched = false;
-                    // next step: one-pass as well (not the first or the diagonal tile), and its S half ready?
+                    // next step: one-pass as well (not the diagonal tile), and its S half ready?
                     const int jn = (u + 1) >> 1, hn = (u + 1) & 1;
                     const bool next_fast = u + 1 < n_steps && jn != k_t;
                     auto late = [&]() {
@@ -641,7 +641,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (lane == 0) { atomicAdd(&cx.status[22], 1); if (redo) atomicAdd(&cx.status[20], 1); }
 #endif
                 if (redo) {
-                    // Generic two-pass form: first and diagonal tiles, steps that move the maximum, and
+                    // Generic two-pass form: the very first step, the diagonal tile, steps that move the maximum, and
                     // every step in debug mode.  The raw accumulators are (still) in tensor memory.
                     uint32_t s[TH];
 #pragma unroll
