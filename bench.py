@@ -482,6 +482,28 @@ def main():
         fl = 4.0 * w.heads * w.head_dim * (float(Lq) * off + float(Lq) ** 2 / 2.0)
         line["chunk"] = {"chunk_len": Lq, "context_len": w.seqlen, "attention_ms": ms,
                          "tflops": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s"}
+    if world == 1 and not args.no_varlen and w.tile == 128 and w.head_dim == 128:
+        # on-the-fly operand mode: no INT8 copies of Q and K and no scales in device memory; the kernel makes
+        # them in shared memory (same mask, same result bit for bit -- checked here on the full workload)
+        po = tm.problem(w.batch, w.heads, w.heads, w.seqlen, w.head_dim, w.tile, w.tile, w.group,
+                        mask_batch=w.mask_batch, flags=tm.QUANT_ON_THE_FLY)
+        q8f, k8f, qsf, ksf = tm.tilemix_quantize_qk(p, qd, kd)
+        words_f, _ = tm.tilemix_pack_routing_mask(p, rd, w.pin_diagonal)
+        ref = tm.tilemix_attention_fwd(p, qd, kd, vd, q8f, k8f, qsf, ksf, words_f, workspace=work)["out"]
+        oo = torch.empty_like(ref)
+        for _ in range(2):
+            tm.tilemix_attention_fwd(po, qd, kd, vd, None, None, None, None, words_f, out=oo, workspace=work)
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        o0.record(stream)
+        for _ in range(3):
+            tm.tilemix_attention_fwd(po, qd, kd, vd, None, None, None, None, words_f, out=oo, workspace=work)
+        o1.record(stream)
+        torch.cuda.synchronize()
+        ms = o0.elapsed_time(o1) / 3
+        line["on_the_fly"] = {"attention_ms": ms, "tflops": F / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                              "equals_quantize_once": bool(torch.equal(oo.view(torch.int16), ref.view(torch.int16))),
+                              "int8_scratch_bytes_saved": int(q8f.numel() + k8f.numel() + 4 * (qsf.numel() + ksf.numel()))}
+        del q8f, k8f, ref, oo
     if world == 1 and not args.no_cpu_baseline:
         dt, pairs, n_rows, threads = oracle_sample(w.scaled(heads=1, batch=1), q, k, v, route, args.cpu_pairs)
         line["cpu_baseline"] = {"value": 4.0 * w.head_dim * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": threads,

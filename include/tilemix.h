@@ -43,6 +43,12 @@ extern "C" {
 /* flags of tilemix_problem_t */
 #define TILEMIX_FORCE_FP16 1u /* ignore the mask: every tile takes the FP16 route; the INT8
                                  operands, scales and mask may then be NULL               */
+#define TILEMIX_QUANT_ON_THE_FLY 2u /* tilemix_attention_fwd, _chunk and tilemix_prefill_host (App. D, the "fused on-the-fly" operand
+                                      mode): q_i8, k_i8, q_scale and k_scale are not read and may be NULL;
+                                      the kernel makes the INT8 tiles and their scales in shared memory from
+                                      the FP16 tiles, for the key tiles routed to INT8 only, with the
+                                      arithmetic of tilemix_quantize_qk -- same result, bit for bit, no INT8
+                                      scratch in device memory.  128x128 tiles with head_dim 128.          */
 /* pack_flags of tilemix_pack_routing_mask */
 #define TILEMIX_PIN_DIAGONAL_FP16 1u
 

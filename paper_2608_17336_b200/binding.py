@@ -14,6 +14,7 @@ LIB_PATH = os.environ.get("TILEMIX_LIB", os.path.join(_HERE, "libtilemix.so"))  
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_WORKSPACE, ERR_DEVICE_TIMEOUT = -1, -2, -3, -4, -5, -6
 FORCE_FP16 = 1
+QUANT_ON_THE_FLY = 2   # flags: INT8 tiles and scales are made inside the attention kernel
 PIN_DIAGONAL_FP16 = 1
 
 EXPORTS = (

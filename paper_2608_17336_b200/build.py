@@ -13,7 +13,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.environ.get("TILEMIX_LIB", os.path.join(HERE, "libtilemix.so"))
 SOURCES = ["api.cu", "varlen.cu", "decode.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu"]
-HEADERS = ["common.cuh", "ptx_sm100.cuh", "softmax_tile.cuh"]
+HEADERS = ["common.cuh", "ptx_sm100.cuh", "softmax_tile.cuh", "quant8.cuh"]
 
 
 def _nvcc() -> str:

@@ -118,7 +118,10 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
     if (rc) return rc;
     if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
     const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
-    if (!force16 && !(q_i8 && k_i8 && q_scale && k_scale && mask_words)) return TILEMIX_ERR_NULL;
+    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;   // INT8 operands and scales are made on chip
+    if (!force16 && !otf && !(q_i8 && k_i8 && q_scale && k_scale)) return TILEMIX_ERR_NULL;
+    if (!force16 && !mask_words) return TILEMIX_ERR_NULL;
+    if (otf && !(g.d == 128 && g.tile_m == 128 && g.tile_n == 128)) return TILEMIX_ERR_UNSUPPORTED;
     if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
     if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
     const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
@@ -159,7 +162,10 @@ int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, cons
     g.W = static_cast<int>(ceil_div(g.T_mask, 32));
     if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
     const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
-    if (!force16 && !(q_i8 && k_i8 && q_scale && k_scale && mask_words)) return TILEMIX_ERR_NULL;
+    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;
+    if (!force16 && !otf && !(q_i8 && k_i8 && q_scale && k_scale)) return TILEMIX_ERR_NULL;
+    if (!force16 && !mask_words) return TILEMIX_ERR_NULL;
+    if (otf && !(g.d == 128 && g.tile_m == 128 && g.tile_n == 128)) return TILEMIX_ERR_UNSUPPORTED;
     if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
     if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
     const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
@@ -339,7 +345,9 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
         int8_t* k8 = reinterpret_cast<int8_t*>(base + a.k8) + k_off;
         float* qs = reinterpret_cast<float*>(base + a.qs) + qs_off;
         float* ks = reinterpret_cast<float*>(base + a.ks) + ks_off;
-        if ((rc = tilemix_quantize_qk(&sub, base + a.q + q_off * 2, base + a.k + k_off * 2, q8, k8, qs, ks, stream)))
+        // (the on-the-fly operand mode has no quantiser pass: the attention kernel ignores q8 .. ks)
+        if (!(g.flags & TILEMIX_QUANT_ON_THE_FLY) &&
+            (rc = tilemix_quantize_qk(&sub, base + a.q + q_off * 2, base + a.k + k_off * 2, q8, k8, qs, ks, stream)))
             return rc;
         if ((rc = tilemix_attention_fwd(&sub, base + a.q + q_off * 2, base + a.k + k_off * 2, base + a.v + k_off * 2, q8, k8,
                                         qs, ks, reinterpret_cast<uint32_t*>(base + a.words) + words_off,

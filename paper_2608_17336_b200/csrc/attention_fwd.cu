@@ -8,9 +8,12 @@
 //   warp  8     TMA producer     (one thread): Q16/Q8 once, then per key tile the K operand(s)
 //                                the routing bits ask for (FP16 and/or INT8) and V, into a
 //                                ring of equally sized shared-memory chunks
-//   warp  9     MMA issuer       (one thread): tcgen05.mma kind::f16 or kind::i8 for S = Q K^T
-//                                per the routing bit, then kind::f16 for O += P V with P read
-//                                from tensor memory; also owns the TMEM allocation
+//   warps 9, 10 MMA issuers      (one thread per query tile): tcgen05.mma kind::f16 or kind::i8 for
+//                                S = Q K^T per the routing bit, then kind::f16 for O += P V with P read
+//                                from tensor memory; warp 9 also owns the TMEM allocation
+//   warp  11    idle, or -- in the on-the-fly operand mode -- the on-chip quantiser: it makes the INT8
+//                                copies of the query tiles and of the key tiles routed to INT8 in
+//                                shared memory from the FP16 tiles (no INT8 operands in global memory)
 // Tensor memory: S_A | S_B | O_A | O_B (FP32 / INT32 accumulators); the FP16 probabilities P
 // overwrite the first half of their S columns.  The two groups alternate: while group A turns
 // S_A into P_A on the ALUs, the tensor pipe runs PV_B and the next QK_B, and vice versa.
@@ -22,6 +25,7 @@
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "quant8.cuh"
 #include "softmax_tile.cuh"
 
 namespace tilemix {
@@ -31,6 +35,7 @@ namespace {
 constexpr int kWarpsPerGroup = 4;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
+constexpr int kQuantWarp = 11;          // on-chip quantiser of the on-the-fly mode (idle otherwise)
 constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
 constexpr int kRegsSoftmax = 216, kRegsOther = 72;   // setmaxnreg split: 2*128*216 + 128*72 = 64512 of the 65536 registers
 constexpr int kRing = 8;
@@ -50,8 +55,9 @@ constexpr float kLn2 = 0.6931471805599453f;
 // touching probabilities already computed, and one pass over O serves all 32 rows.
 constexpr float kTauSoft = 8.0f, kTauHard = 15.0f, kMargin = 6.0f;
 
-enum Role : int { kRoleSoftmaxA = 0, kRoleSoftmaxB = 1, kRoleProducer = 2, kRoleMma = 3 };
-enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6, kBarPV = 7 };
+enum Role : int { kRoleSoftmaxA = 0, kRoleSoftmaxB = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQuant = 4 };
+enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6, kBarPV = 7,
+                 kBarRaw = 8, kBarQ8 = 9 };
 
 template <int D, int T>
 struct Cfg {
@@ -73,9 +79,9 @@ struct Cfg {
     static constexpr int kOffRing = kOffQ8 + 2 * kQ8Tile;
     static constexpr int kOffBars = kOffRing + kRing * kChunk;
     static constexpr int kTH = T / 2;                 // key columns per half step
-    static constexpr int kNumBars = 2 + 2 * kRing + 4 + 4 + 2 + 2 + 1;
-    static constexpr int kOffMisc = kOffBars + kNumBars * 8;       // tmem base, abort flag
-    static constexpr int kOffWords = kOffMisc + 16;
+    static constexpr int kNumBars = 2 + 2 * kRing + 4 + 4 + 2 + 2 + 1 + kBundles + 2;
+    static constexpr int kOffMisc = kOffBars + kNumBars * 8;       // tmem base, abort flag; on-chip scales
+    static constexpr int kOffWords = kOffMisc + 64;
     static constexpr int kSmemBytes = kOffWords + kMaxTiles / 2;   // 4-bit schedule entries
     static constexpr int kSmemAlloc = kSmemBytes + 1024;           // slack to align the base
     static_assert(kK8Bytes <= kChunk, "INT8 key tile must fit one ring chunk");
@@ -153,7 +159,7 @@ __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t p
         }
     }
 #ifdef TILEMIX_PHASE_TIMERS
-    if ((threadIdx.x & 127) == 0 || role >= kRoleProducer) TM_TIMER_ADD(role * 8 + which, clock64() - c0);
+    if ((threadIdx.x & 127) == 0 || role >= kRoleProducer) TM_TIMER_ADD((role & 3) * 8 + (which & 7), clock64() - c0);
 #endif
     return true;
 }
@@ -174,7 +180,10 @@ struct Ring {
 };
 
 // VL: variable-length batch (the work item is found in the sequence prefix sums).
-template <int D, int T, bool VL>
+// OTF: on-the-fly operand generation (App. D, "fused on-the-fly" mode): there are no INT8 copies of Q and K
+// and no scales in global memory; a quantiser warp makes them in shared memory from the FP16 tiles, for
+// the key tiles some query tile of the CTA routes to INT8 only.
+template <int D, int T, bool VL, bool OTF>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                  const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16,
@@ -242,7 +251,16 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     auto bar_pv = [&](int t) { return bar0 + 8u * (10 + 2 * kRing + t); };   // every PV of tile t
     auto bar_o = [&](int t) { return bar0 + 8u * (12 + 2 * kRing + t); };    // the last PV of tile t
     const uint32_t bar_drain = bar0 + 8u * (14 + 2 * kRing);
+    // on-the-fly mode: "FP16 K tile of bundle i landed and its INT8 chunk is free" (producer -> quantiser),
+    // "INT8 copy and scale of query tile t are in shared memory" (quantiser -> issuers, softmax groups)
+    auto bar_raw = [&](int i) { return bar0 + 8u * (15 + 2 * kRing + i); };
+    auto bar_q8 = [&](int t) { return bar0 + 8u * (15 + 2 * kRing + kBundles + t); };
     uint32_t* misc = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);   // [0] tmem base, [1] abort
+    // on-the-fly mode: delta_K of bundle n at otf_dk[n % (2 kBundles)] (a slot is rewritten only after
+    // bundle n + kBundles has been consumed, i.e. long after both groups finished key tile n), delta_Q of
+    // query tile t at otf_dq[t]
+    volatile float* otf_dk = reinterpret_cast<volatile float*>(misc + 4);
+    volatile float* otf_dq = reinterpret_cast<volatile float*>(misc + 12);
     uint32_t* sched_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
     Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status};
 
@@ -250,9 +268,14 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         ptx::mbar_init(bar_q(0), 1);
         ptx::mbar_init(bar_q(1), 1);
         for (int i = 0; i < kBundles; ++i) {
-            ptx::mbar_init(bar_full(i), 1);
+            // on-the-fly mode: a second arrival, by the quantiser (after it made the bundle's INT8 tile, if
+            // there is one to make)
+            ptx::mbar_init(bar_full(i), OTF ? 2 : 1);
             ptx::mbar_init(bar_empty(i), hasB ? 2 : 1);   // one arrival per MMA issuer
+            ptx::mbar_init(bar_raw(i), 2);                // K16 bytes expected + "INT8 chunk claimed"
         }
+        ptx::mbar_init(bar_q8(0), 1);
+        ptx::mbar_init(bar_q8(1), 1);
         for (int t = 0; t < 2; ++t) {
             for (int h = 0; h < 2; ++h) {
                 ptx::mbar_init(bar_s(t, h), 1);
@@ -284,6 +307,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const bool useA = j <= kA;
             if ((useA && !(e & 1u)) || (hasB && !(e & 2u))) e |= 4u;
             if ((useA && (e & 1u)) || (hasB && (e & 2u))) e |= 8u;
+            if (OTF && (e & 8u)) e |= 4u;   // the INT8 copy is made from the FP16 tile
             packed |= e << (4 * jj);
         }
         sched_s[i] = packed;
@@ -298,7 +322,99 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const uint32_t tmem_base = misc[0];
     auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
-    if (warp >= kMmaWarp + 2 || (warp == kMmaWarp + 1 && !hasB)) {
+    if (OTF && warp == kQuantWarp) {
+        // ================================================================ on-chip quantiser (on-the-fly mode)
+        // One warp makes the INT8 copies the tensor pipe reads: of the two query tiles once, then of every
+        // key tile some query tile of the CTA routes to INT8.  A tile is 128 rows = one quantisation block
+        // (App. C): delta = max|x| / 127 over the tile, codes by the quantiser's own arithmetic.  Source and
+        // destination are the shared-memory images TMA would have written: FP16 tiles as D/64 slabs of
+        // 128-byte rows, INT8 tiles as 128-byte rows, both with the 128-byte swizzle (16-byte chunk c of row r
+        // sits at chunk c ^ (r & 7)).
+        ptx::setmaxnreg_dec<kRegsOther>();
+        static_assert(!OTF || (D == 128 && T == 128), "the on-chip quantiser handles 128 x 128 tiles");
+        bool ok = true;
+        auto quantise_tile = [&](uint32_t src_off, uint32_t dst_off) -> float {
+            const uint8_t* src = smem + src_off;
+            uint8_t* dst = smem + dst_off;
+            constexpr int kVec = C::kHalves * 128 * 8;   // 16-byte vectors (8 elements) of the FP16 tile
+            uint32_t amax2 = 0u;
+            for (int i0 = lane; i0 < kVec; i0 += 32 * 8) {   // eight loads in flight per lane
+                uint4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const uint4*>(src + (i0 + 32 * u) * 16);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    amax2 = umax2(amax2, umax2(umax2(habs2_bits(v[u].x), habs2_bits(v[u].y)),
+                                               umax2(habs2_bits(v[u].z), habs2_bits(v[u].w))));
+            }
+            uint32_t amax = max(amax2 & 0xffffu, amax2 >> 16);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            const float amax_f = __half2float(__ushort_as_half(static_cast<unsigned short>(amax)));
+            const float delta = __fdiv_rn(amax_f, 127.0f);
+            if (amax == 0u) {   // zero block: delta = 0, every code 0
+                for (int i = lane; i < 128 * D / 16; i += 32)
+                    *reinterpret_cast<uint4*>(dst + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+                return delta;
+            }
+            const float rdelta = __frcp_rn(delta);
+            for (int i0 = lane; i0 < kVec; i0 += 32 * 4) {   // four vectors in flight per lane
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const uint4*>(src + (i0 + 32 * u) * 16);
+                uint2 qv[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) qv[u] = quant8_div(v[u], delta, rdelta);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + 32 * u;
+                    const int slab = i >> 10, r = (i >> 3) & 127, cl = (i & 7) ^ (r & 7);   // logical chunk of the slab
+                    // elements 64 slab + 8 cl .. + 7 of row r: byte column 64 slab + 8 cl of the INT8 row
+                    const int c16 = slab * 4 + (cl >> 1);
+                    *reinterpret_cast<uint2*>(dst + r * 128 + ((c16 ^ (r & 7)) << 4) + (cl & 1) * 8) = qv[u];
+                }
+            }
+            return delta;
+        };
+        // hand-over to the async proxy (the tensor pipe reads shared memory through it), then one arrival
+        auto publish = [&](uint32_t bar) {
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar);
+        };
+        // The quantiser arrives on the "landed" barrier of EVERY bundle, with or without an INT8 tile to
+        // make, so that the issuers (and with them the producer) can never run more than kBundles bundles
+        // ahead of it and the phase it waits for is unambiguous.  A query tile is quantised just before the
+        // first key tile it routes to INT8.
+        Ring ring;   // the producer's sequence of chunks
+        uint32_t q8_made = 0u;
+        for (int n = 0; n < nkv && ok; ++n) {
+            const uint32_t e = sched(n);
+            uint32_t s16 = 0, s8 = 0;
+            if (n >= 1) ring.take(C::kHalves);
+            if (e & 4u) s16 = ring.take(C::kHalves);
+            if (e & 8u) s8 = ring.take(1);
+            for (int t = 0; t < 2; ++t) {
+                if (!((e >> t) & 1u) || ((q8_made >> t) & 1u)) continue;
+                ok = wait_bar(cx, bar_q(t), 0, kRoleQuant, t, kBarQ);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const float dq = quantise_tile(C::kOffQ16 + t * C::kQ16Tile, C::kOffQ8 + t * C::kQ8Tile);
+                if (lane == 0) otf_dq[t] = dq;
+                publish(bar_q8(t));
+                q8_made |= 1u << t;
+            }
+            if (!ok) break;
+            ok = wait_bar(cx, bar_raw(n % kBundles), (n / kBundles) & 1, kRoleQuant, n, kBarRaw);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (e & 8u) {
+                const float dk = quantise_tile(C::kOffRing + s16 * C::kChunk, C::kOffRing + s8 * C::kChunk);
+                if (lane == 0) otf_dk[n % (2 * kBundles)] = dk;
+            }
+            publish(bar_full(n % kBundles));
+        }
+    } else if (warp >= kMmaWarp + 2 || (warp == kMmaWarp + 1 && !hasB)) {
         ptx::setmaxnreg_dec<kRegsOther>();   // idle warps of the third warpgroup
     } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer
@@ -307,18 +423,18 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             ptx::tma_prefetch_desc(&tm_q16);
             ptx::tma_prefetch_desc(&tm_k16);
             ptx::tma_prefetch_desc(&tm_v16);
-            if (prm.has_int8) {
+            if (prm.has_int8 && !OTF) {
                 ptx::tma_prefetch_desc(&tm_q8);
                 ptx::tma_prefetch_desc(&tm_k8);
             }
             for (int t = 0; t < (hasB ? 2 : 1); ++t) {
                 const int m = t ? mB : mA;
-                const uint32_t bytes = C::kQ16Tile + (prm.has_int8 ? C::kQ8Tile : 0);
+                const uint32_t bytes = C::kQ16Tile + ((prm.has_int8 && !OTF) ? C::kQ8Tile : 0);
                 ptx::mbar_arrive_expect_tx(bar_q(t), bytes);
                 for (int c = 0; c < C::kHalves; ++c)
                     ptx::tma_load_4d(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, &tm_q16,
                                      bar_q(t), c * 64, tok0 + m * T, hq, b);
-                if (prm.has_int8)
+                if (prm.has_int8 && !OTF)
                     ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
             }
             // Chunks are taken from the ring in the order K16_j?, K8_j?, V_j (j = 0, 1, ...), the same
@@ -340,17 +456,28 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 // bundle n: V of key tile n - 1 (n >= 1) and the K copies of key tile n (n < nkv)
                 const uint32_t e = n < nkv ? sched(n) : 0u;
                 const bool has_v = n >= 1;
-                uint32_t s16 = 0, s8 = 0, sv = 0, bytes = 0;
+                uint32_t s16 = 0, s8 = 0, sv = 0, bytes = 0, raw_bytes = 0;
+                // On-the-fly mode: the FP16 K tile of a bundle with an INT8 tile to make is announced to the
+                // quantiser (bar_raw), not to the issuers; the INT8 chunk is only claimed, not filled.
+                const bool make8 = OTF && (e & 8u);
                 // chunk order inside the sequence: ..., V_{n-1}, K16_n, K8_n, V_n, ...
                 if (has_v) { sv = ring.take(C::kHalves); bytes += C::kHalves * C::kChunk; }
-                if (e & 4u) { s16 = ring.take(C::kHalves); bytes += C::kHalves * C::kChunk; }
-                if (e & 8u) { s8 = ring.take(1); bytes += C::kK8Bytes; }
-                if (bytes == 0u) break;             // nothing after the last V
+                if (e & 4u) { s16 = ring.take(C::kHalves); (make8 ? raw_bytes : bytes) += C::kHalves * C::kChunk; }
+                if (e & 8u) { s8 = ring.take(1); if (!OTF) bytes += C::kK8Bytes; }
+                if (bytes == 0u && raw_bytes == 0u) break;             // nothing after the last V
                 if (n >= kBundles) wait_consumed(n - kBundles, n);     // its barriers are free again
                 // the barrier is armed for the whole bundle first; every operand is then copied as soon as
                 // its own chunks are free, so a V tile does not wait for the room of the K tile behind it
                 const uint32_t bar = bar_full(n % kBundles);
-                ptx::mbar_arrive_expect_tx(bar, bytes);
+                if (bytes != 0u) ptx::mbar_arrive_expect_tx(bar, bytes);
+                else ptx::mbar_arrive(bar);
+                if (OTF) {
+                    if (n == nkv) ptx::mbar_arrive(bar);   // the last bundle (V only) is not the quantiser's
+                    if (n < nkv) {
+                        if (raw_bytes != 0u) ptx::mbar_arrive_expect_tx(bar_raw(n % kBundles), raw_bytes);
+                        else ptx::mbar_arrive(bar_raw(n % kBundles));
+                    }
+                }
                 armed = n + 1;
                 auto claim = [&](uint32_t slot, int chunks) {
                     for (int c = 0; c < chunks; ++c) {
@@ -367,20 +494,27 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (e & 4u) {
                     claim(s16, C::kHalves);
                     if (!ok) break;
+                    const uint32_t bar16 = make8 ? bar_raw(n % kBundles) : bar;
                     for (int c = 0; c < C::kHalves; ++c)
-                        ptx::tma_load_4d(sbase + C::kOffRing + (s16 + c) * C::kChunk, &tm_k16, bar, c * 64, tok0 + n * T, hk, b);
+                        ptx::tma_load_4d(sbase + C::kOffRing + (s16 + c) * C::kChunk, &tm_k16, bar16, c * 64, tok0 + n * T, hk, b);
                 }
                 if (e & 8u) {
                     claim(s8, 1);
                     if (!ok) break;
-                    ptx::tma_load_4d(sbase + C::kOffRing + s8 * C::kChunk, &tm_k8, bar, 0, tok0 + n * T, hk, b);
+                    if (!OTF) ptx::tma_load_4d(sbase + C::kOffRing + s8 * C::kChunk, &tm_k8, bar, 0, tok0 + n * T, hk, b);
                 }
+                // on-the-fly mode, second arrival: the INT8 chunk (if any) is the quantiser's to write
+                if (OTF && n < nkv) ptx::mbar_arrive(bar_raw(n % kBundles));
             }
             if (!ok || *cx.abort_flag) {
                 // let copies that are still in flight land before the CTA's memory is released
-                for (int n = armed > kBundles ? armed - kBundles : 0; n < armed; ++n)
+                for (int n = armed > kBundles ? armed - kBundles : 0; n < armed; ++n) {
                     for (int it = 0; it < (1 << 20); ++it)
                         if (ptx::mbar_try_wait(bar_full(n % kBundles), (n / kBundles) & 1)) break;
+                    if (OTF && n < nkv)
+                        for (int it = 0; it < (1 << 20); ++it)
+                            if (ptx::mbar_try_wait(bar_raw(n % kBundles), (n / kBundles) & 1)) break;
+                }
             }
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
@@ -397,6 +531,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             constexpr uint32_t kIdescPV = ptx::instr_desc(1, 0, 0, 1, C::kM, D);
             Ring ring;
             bool ok = true;
+            bool q8_there = !OTF;   // on-the-fly mode: the INT8 copy of Q is waited for before its first use
             // Wait until bundle n has landed.  An issuer waits for EVERY bundle, also one whose data it
             // does not read: its arrival on the bundle's "consumed" barrier must not run a round of the
             // barriers ahead of the other issuer's, or two arrivals of one issuer would release it.
@@ -417,6 +552,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             auto issue_qk = [&](int t, int h, uint32_t int8_route, uint32_t s16, uint32_t s8) {
                 const uint32_t d_tmem = tmem_base + t * C::kSCols + h * TH;
                 if (int8_route) {
+                    if constexpr (OTF) {
+                        if (!q8_there) {
+                            if (!wait_bar(cx, bar_q8(t), 0, kRoleMma, t, kBarQ8)) { ok = false; return; }
+                            q8_there = true;
+                        }
+                    }
                     const uint32_t a_lo = ptx::desc_lo(sbase + C::kOffQ8 + t * C::kQ8Tile, 16);
                     const uint32_t b_lo = ring_lo + s8 * kChunkLo + ((h * TH * C::kI8RowBytes) >> 4);
                     ptx::mma_i8_ss<false>(d_tmem, a_lo, kHi8, b_lo, kHi8, kIdescQK8);
@@ -526,21 +667,26 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const bool row_valid = row < T && i_loc < len;
             // scales: dense [B,H,T_m] (unit stride over blocks), variable-length [blocks, H]
             const int64_t dk_step = varlen ? prm.Hk : 1;
-            const float dq = !prm.has_int8 ? 0.f
-                             : varlen ? prm.q_scale[static_cast<int64_t>(row0 + m_t) * prm.Hq + hq]
-                                      : prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t];
-            const float* dk_row = !prm.has_int8 ? nullptr
-                                  : varlen ? prm.k_scale + static_cast<int64_t>(row0) * prm.Hk + hk
-                                           : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.ks_blocks;
+            float dq = 0.f;
+            const float* dk_row = nullptr;
+            if constexpr (!OTF) {
+                if (prm.has_int8) {
+                    dq = varlen ? prm.q_scale[static_cast<int64_t>(row0 + m_t) * prm.Hq + hq]
+                                : prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t];
+                    dk_row = varlen ? prm.k_scale + static_cast<int64_t>(row0) * prm.Hk + hk
+                                    : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.ks_blocks;
+                }
+            }
             float m_run = -INFINITY, z = 0.f;
             float m_seen = -INFINITY;     // largest scaled score seen so far (m_run may lag it)
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
+            bool dq_there = !OTF;   // on-the-fly mode: this tile's scale comes from the on-chip quantiser
 
 #ifdef TILEMIX_PHASE_TIMERS
             const long long loop_c0 = clock64();
 #endif
-            float dk_next = prm.has_int8 ? dk_row[0] : 0.f;
+            float dk_next = (prm.has_int8 && !OTF) ? dk_row[0] : 0.f;
             float a = prm.scale_log2;
             uint32_t int8_route = 0u;
             constexpr int TH = C::kTH;
@@ -561,7 +707,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         a *= dq * dk_next;
                         if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                     }
-                    if (prm.has_int8 && j < k_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
+                    if (!OTF && prm.has_int8 && j < k_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
                 }
                 const uint32_t t_sh = t_s + h * TH;
 #ifdef TILEMIX_PHASE_TIMERS
@@ -572,6 +718,21 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
+                }
+                if constexpr (OTF) {
+                    // the key tile's scale was written by the quantiser before the issuer could start the
+                    // MMAs whose result has just been seen
+                    if (h == 0 && int8_route) {
+                        if (!dq_there) {
+                            ok = wait_bar(cx, bar_q8(t), 0, role, m_t, kBarQ8);   // long over: S of an INT8 tile is there
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            dq = otf_dq[t];
+                            dq_there = true;
+                        }
+                        a = prm.scale_log2 * (dq * otf_dk[j % (2 * kBundles)]);   // same rounding order as with scales from memory
+                        if (a == 0.f) a = 1.f;
+                    }
                 }
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(39, clock64() - sw0);
@@ -840,12 +1001,14 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     EncodeTiledFn enc = nullptr;
     int rc = get_encoder(&enc);
     if (rc) return rc;
-    const bool has8 = !(g.flags & TILEMIX_FORCE_FP16) && q8 != nullptr;
+    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;
+    if (otf && (vl != nullptr || !(D == 128 && T == 128))) return TILEMIX_ERR_UNSUPPORTED;
+    const bool has8 = !(g.flags & TILEMIX_FORCE_FP16) && (q8 != nullptr || otf);
     CUtensorMap tq, tk, tv, tq8, tk8;
     if ((rc = encode_map(enc, &tq, q, 2, g.d, g.L, g.Hq, g.B, g.qs, 64, C::kM, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
     if ((rc = encode_map(enc, &tk, k, 2, g.d, g.Lk, g.Hk, g.B, g.ks, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
     if ((rc = encode_map(enc, &tv, v, 2, g.d, g.Lk, g.Hk, g.B, g.vs, 64, T, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
-    if (has8) {
+    if (has8 && !otf) {
         const CUtensorMapSwizzle sw8 = (D == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
         const int64_t dq[3] = {static_cast<int64_t>(g.Hq) * g.L * g.d, static_cast<int64_t>(g.L) * g.d, g.d};
         const int64_t dk[3] = {static_cast<int64_t>(g.Hk) * g.Lk * g.d, static_cast<int64_t>(g.Lk) * g.d, g.d};
@@ -876,7 +1039,10 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     }
     cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceClearBytes, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
-    const auto kernel = vl ? attention_kernel<D, T, true> : attention_kernel<D, T, false>;
+    auto kernel = vl ? attention_kernel<D, T, true, false> : attention_kernel<D, T, false, false>;
+    if constexpr (D == 128 && T == 128) {
+        if (otf) kernel = attention_kernel<D, T, false, true>;
+    }
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
     if (e != cudaSuccess) return static_cast<int>(e);
     const int64_t ctas = vl ? static_cast<int64_t>(g.Hq) * total_pairs

@@ -180,6 +180,7 @@ int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varle
     int rc = resolve_varlen(p, vl, &g, &t);
     if (rc) return rc;
     if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
+    if ((g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0) return TILEMIX_ERR_UNSUPPORTED;   // dense batches only
     const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
     if (!force16 && !(q_i8 && k_i8 && q_scale && k_scale && mask_words)) return TILEMIX_ERR_NULL;
     if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;

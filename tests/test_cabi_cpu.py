@@ -72,6 +72,20 @@ def test_host_side_validation_without_gpu(lib):
     dbg = b.DebugStruct(None, 3, None, None)
     assert lib.tilemix_attention_fwd(ctypes.byref(good), *_args(9), None, ctypes.c_void_p(0x1000), 4096,
                                      ctypes.byref(dbg), None) == b.ERR_NULL
+    # on-the-fly operand mode: the INT8 operands and scales may be NULL (the call gets as far as the workspace
+    # check), the routing words may not; 128x128 tiles only
+    one = ctypes.c_void_p(0x1000)
+    otf = b.problem(1, 2, 2, 1024, 128, 128, 128, flags=b.QUANT_ON_THE_FLY)
+    assert lib.tilemix_attention_fwd(ctypes.byref(otf), one, one, one, None, None, None, None, one, one, None,
+                                     one, 8, None, None) == b.ERR_WORKSPACE
+    assert lib.tilemix_attention_fwd(ctypes.byref(otf), one, one, one, None, None, None, None, None, one, None,
+                                     one, 4096, None, None) == b.ERR_NULL
+    otf64 = b.problem(1, 2, 2, 1024, 64, 64, 64, flags=b.QUANT_ON_THE_FLY)
+    assert lib.tilemix_attention_fwd(ctypes.byref(otf64), one, one, one, None, None, None, None, one, one, None,
+                                     one, 4096, None, None) == b.ERR_UNSUPPORTED
+    chunk = b.problem(1, 2, 2, 256, 64, 64, 64, flags=b.QUANT_ON_THE_FLY)
+    assert lib.tilemix_attention_fwd_chunk(ctypes.byref(chunk), 1024, *_args(9), None, one, 4096, None,
+                                           None) == b.ERR_UNSUPPORTED
     assert lib.tilemix_launch_count() == 0
 
 
@@ -163,6 +177,9 @@ def test_varlen_host_side_validation(lib):
                                                 None) == b.ERR_NULL
     assert lib.tilemix_attention_fwd_varlen(ctypes.byref(ok), vl.ref(), one, one, one, None, None, None, None,
                                             None, one, None, one, 8192, None, None) == b.ERR_NULL
+    otf = b.problem(1, 2, 2, 300, 64, 64, 64, flags=b.QUANT_ON_THE_FLY)   # dense batches only
+    assert lib.tilemix_attention_fwd_varlen(ctypes.byref(otf), vl.ref(), one, one, one, one, one, one, one,
+                                            one, one, None, one, 8192, None, None) == b.ERR_UNSUPPORTED
     long = b.problem(1, 1, 1, 64 * 2049, 64, 64, 64, flags=b.FORCE_FP16)
     assert lib.tilemix_attention_fwd_varlen(ctypes.byref(long), b.Varlen([0, 64 * 2049]).ref(), one, one, one,
                                             None, None, None, None, None, one, None, one, 8192, None,
