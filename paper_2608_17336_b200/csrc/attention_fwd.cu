@@ -624,15 +624,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (mine) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-#if defined(TILEMIX_TRACE) && !defined(TILEMIX_TRACE4)
-                        if (blockIdx.x == 5 && j >= 8 && j < 8 + 16)
-                            reinterpret_cast<long long*>(cx.status)[320 + ((j - 8) * 4 + 2 * h + t) * 2 + 1] = clock64();
-#endif
                         if (!wait_bar(cx, bar_p(t, h), j & 1, kRoleMma, j, kBarP)) { ok = false; break; }
-#if defined(TILEMIX_TRACE) && !defined(TILEMIX_TRACE4)
-                        if (blockIdx.x == 5 && j >= 8 && j < 8 + 16)
-                            reinterpret_cast<long long*>(cx.status)[320 + ((j - 8) * 4 + 2 * h + t) * 2] = clock64();
-#endif
                         ptx::tc_fence_after_sync();
                         issue_pv(t, h, sv, (j > 0 || h > 0) ? 1u : 0u);
                         ptx::mma_commit(bar_pv(t));
@@ -740,10 +732,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st0 = clock64();
 #endif
-#ifdef TILEMIX_TRACE
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
-                    reinterpret_cast<long long*>(cx.status)[128 + ((u - 16) * 2 + t) * 2] = clock64();
-#endif
 
                 // ---- shared online-softmax state (Sec. 3.1), log2 domain --------------------------
                 // P = 2^(a*raw - m) is rounded to FP16 and packed two per word into p2[0 .. TH/2).
@@ -760,9 +748,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (__any_sync(0xffffffffu, m_seen > m_run + kTauSoft)) {
                     // Deferred move of the maximum decided on an earlier step (all rows of the warp):
                     // z changes scale here, O~ below together with any move this step itself forces.
-#ifdef TILEMIX_TRACE
-                    if (lane == 0) atomicAdd(&cx.status[21], 1);
-#endif
                     const float m_new = fmaxf(m_run, m_seen + kMargin);
                     alpha = fast_exp2(m_run - m_new);   // 1 for rows that are up to date
                     m_run = m_new;
@@ -794,12 +779,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 }
 #ifdef TILEMIX_PHASE_TIMERS
                 const long long st2 = clock64() + (__float_as_int(sum) & 0);
-#endif
-#ifdef TILEMIX_TRACE4
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
-                    reinterpret_cast<long long*>(cx.status)[320 + ((u - 16) * 2 + t) * 2] = clock64() + (__float_as_int(sum) & 0);
-#elif defined(TILEMIX_TRACE)
-                if (lane == 0) { atomicAdd(&cx.status[22], 1); if (redo) atomicAdd(&cx.status[20], 1); }
 #endif
                 if (redo) {
                     // Generic two-pass form: the very first step, the diagonal tile, steps that move the maximum, and
@@ -888,16 +867,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     ptx::tmem_st16(t_sh, p2);
                 }
                 ptx::tmem_wait_st();
-#ifdef TILEMIX_TRACE4
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
-                    reinterpret_cast<long long*>(cx.status)[320 + ((u - 16) * 2 + t) * 2 + 1] = clock64();
-#endif
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t, h));
-#ifdef TILEMIX_TRACE
-                if (blockIdx.x == 5 && (threadIdx.x & 127) == 0 && u >= 16 && u < 16 + 48)
-                    reinterpret_cast<long long*>(cx.status)[128 + ((u - 16) * 2 + t) * 2 + 1] = clock64();
-#endif
 #ifdef TILEMIX_PHASE_TIMERS
                 if ((threadIdx.x & 127) == 0) {
                     const long long st4 = clock64();

@@ -16,32 +16,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-// 2^x for x <= ~kTau on the FMA pipe (no special-function unit): x = n + f with n = round(x),
-// f in [-0.5, 0.5]; 2^f by a cubic (max relative error 7.5e-5, below the FP16 rounding of P);
-// 2^n by adding n to the exponent field.  Inputs are clamped to >= -126.
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    const float2 magic = make_float2(12582912.f, 12582912.f);       // 1.5 * 2^23
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 r = __fadd2_rn(x, magic);                           // low mantissa bits = round(x)
-    const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
-    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p = __ffma2_rn(f, make_float2(0.055171649903059006f, 0.055171649903059006f),
-                          make_float2(0.2426111251115799f, 0.2426111251115799f));
-    p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
-    p = __ffma2_rn(p, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
-    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
-    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
-    return p;
-}
-
-// Every kPolyEvery-th pair of an interior tile takes the polynomial instead of the special-function
-// unit (0 = none), so that both pipes work on a tile at the same time.
-#ifndef TILEMIX_POLY_EVERY
-#define TILEMIX_POLY_EVERY 0
-#endif
-constexpr int kPolyEvery = TILEMIX_POLY_EVERY;
-
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -93,10 +67,7 @@ __device__ __forceinline__ void softmax_tile_fast(uint32_t t_s, uint32_t (&first
         if (i == kLateAt) late();
         if (i >= kE && i - kE < NP) {                         // exponentials of pair i - kE
             const int k = i - kE;
-            if (kPolyEvery > 0 && (k % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1)
-                eb[k & 7] = exp2_poly2(tb[k & 3]);
-            else
-                eb[k & 7] = make_float2(fast_exp2(tb[k & 3].x), fast_exp2(tb[k & 3].y));
+            eb[k & 7] = make_float2(fast_exp2(tb[k & 3].x), fast_exp2(tb[k & 3].y));
         }
         if (i >= 2 && i - 2 < NP) {                           // a*raw - m of pair i - 2
             const int k = i - 2;
