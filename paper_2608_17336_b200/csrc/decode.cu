@@ -330,7 +330,6 @@ decode_kernel(const DecodeParams prm) {
             // at this lane group's columns of this warp's blocks
             const uint8_t* vbase = vst + (16 * ks + 2 * t) * D + BPG * g + nb0;
             const __half2 off = __floats2half2_rn(1152.f, 1152.f);
-            float dummy[2] = {0.f, 0.f};
 #pragma unroll
             for (int w = 0; w < NBLK / 4; ++w) {
                 // four column blocks at a time: one 32-bit word of each of the four rows
@@ -354,10 +353,11 @@ decode_kernel(const DecodeParams prm) {
                     uint32_t b0 = __byte_perm(s01, 0x64646464u, sel), b1 = __byte_perm(s23, 0x64646464u, sel);
                     const __half2 v0 = __hsub2(*reinterpret_cast<const __half2*>(&b0), off);
                     const __half2 v1 = __hsub2(*reinterpret_cast<const __half2*>(&b1), off);
-                    float c[4] = {acc[4 * w + e][0], acc[4 * w + e][1], dummy[0], dummy[1]};
+                    // rows g + 8 of the product do not exist: their accumulators start at 0 and are dropped, so
+                    // that the MMAs of different column blocks do not depend on one another
+                    float c[4] = {acc[4 * w + e][0], acc[4 * w + e][1], 0.f, 0.f};
                     mma_f16(c, pa0, pa2, *reinterpret_cast<const uint32_t*>(&v0), *reinterpret_cast<const uint32_t*>(&v1));
                     acc[4 * w + e][0] = c[0]; acc[4 * w + e][1] = c[1];
-                    dummy[0] = c[2]; dummy[1] = c[3];
                 }
             }
             if (!counts_z) z_part = 0.f;   // the row sum of a key step is counted by one of its warps
