@@ -153,3 +153,63 @@ def test_on_the_fly_chunked_prefill():
     assert code == 0, rec
     assert torch.equal(res["out"].view(torch.int16), full["out"][:, :, off:].contiguous().view(torch.int16))
     assert torch.equal(res["lse"], full["lse"][:, :, off:])
+
+
+def test_on_the_fly_quantiser_on_ties_and_awkward_scales():
+    """The on-chip quantiser forms the IEEE quotient by refinement instead of a division; the quantise-once kernel
+    falls back to a true division near ties.  Inputs that sit exactly on ties (x / delta = k + 1/2), one binary16
+    step next to them, and blocks whose maximum gives awkward reciprocals must come out the same, code for code:
+    checked through the raw INT32 accumulators of every tile and the outputs."""
+    from paper_2608_17336_b200 import binding as tm
+    L, d, H = 512, 128, 2
+    rng = np.random.default_rng(66)
+    def block(amax, kind):
+        x = np.zeros((128, d), np.float16)
+        ks = rng.integers(0, 127, size=(128, d)).astype(np.float32)
+        sign = rng.choice([-1.0, 1.0], size=(128, d)).astype(np.float32)
+        delta = np.float32(amax) / np.float32(127)
+        if kind == "tie":            # exact ties when delta is a power of two times something exact in binary16
+            v = (ks + 0.5) * delta
+        elif kind == "near":         # one binary16 step above / below a tie
+            v = np.nextafter(((ks + 0.5) * delta).astype(np.float16), np.float16(np.inf) * rng.choice([-1, 1], size=(128, d)).astype(np.float16)).astype(np.float32)
+        else:
+            v = rng.standard_normal((128, d)).astype(np.float32) * amax / 4
+        x[:] = np.clip(sign * v, -amax, amax).astype(np.float16)
+        x[0, 0] = np.float16(amax)   # pins the block maximum
+        return x
+    recipe = [(127.0, "tie"), (63.5, "tie"), (127.0, "near"), (1.0, "near"), (3.0, "rand"), (0.3337, "near"),
+              (1000.0, "tie"), (6.1e-5, "rand")]
+    def tensor():
+        t = np.zeros((1, H, L, d), np.float16)
+        for h in range(H):
+            for blk in range(L // 128):
+                amax, kind = recipe[(h * 4 + blk) % len(recipe)]
+                t[0, h, blk * 128:(blk + 1) * 128] = block(amax, kind)
+        return torch.from_numpy(t)
+    q, k = tensor(), tensor()
+    v = torch.from_numpy(rng.standard_normal((1, H, L, d)).astype(np.float16))
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    p = tm.problem(1, H, H, L, d, 128, 128, 1, softmax_scale=1e-4)
+    q8, k8, qs, ks_ = tm.tilemix_quantize_qk(p, qd, kd)
+    route = np.ones((1, H, p.T_m, p.T_mask), np.uint8)
+    words, _ = tm.tilemix_pack_routing_mask(p, torch.from_numpy(route).to(dev), False)
+    tiles = [(0, h, m, n) for h in range(H) for m in range(4) for n in range(m + 1)]
+    once = tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks_, words, debug_tiles=tiles)
+    po = tm.problem(1, H, H, L, d, 128, 128, 1, softmax_scale=1e-4, flags=tm.QUANT_ON_THE_FLY)
+    otf = tm.tilemix_attention_fwd(po, qd, kd, vd, None, None, None, None, words, debug_tiles=tiles)
+    assert tm.tilemix_read_status(otf["workspace"])[0] == 0
+    assert torch.equal(otf["raw"], once["raw"])
+    assert torch.equal(otf["out"].view(torch.int16), once["out"].view(torch.int16))
+    # and the codes are the definition's: raw accumulators against the oracle quantiser
+    import oracle
+    q8o, _ = oracle.quantize(H_np(q), 128)
+    k8o, _ = oracle.quantize(H_np(k), 128)
+    raw = otf["raw"].cpu().numpy()
+    for e, (b, h, m, n) in enumerate(tiles):
+        want = q8o[b, h, m * 128:(m + 1) * 128].astype(np.int32) @ k8o[b, h, n * 128:(n + 1) * 128].astype(np.int32).T
+        assert np.array_equal(raw[e], want), (h, m, n)
+
+
+def H_np(t):
+    return H.np_bits(t)
