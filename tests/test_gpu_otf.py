@@ -213,3 +213,19 @@ def test_on_the_fly_quantiser_on_ties_and_awkward_scales():
 
 def H_np(t):
     return H.np_bits(t)
+
+
+def test_on_the_fly_with_the_mask_ignored():
+    """TILEMIX_FORCE_FP16 on top of the on-the-fly flag: nothing is quantised, the result is the all-FP16 one."""
+    from paper_2608_17336_b200 import binding as tm
+    w = synth.Workload("otf16", 1, 2, 700, 128, 128, 1, seed=67)
+    q, k, v = synth.make_qkv(w)
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    outs = []
+    for flags in (tm.FORCE_FP16, tm.FORCE_FP16 | tm.QUANT_ON_THE_FLY):
+        p = tm.problem(1, 2, 2, 700, 128, 128, 128, 1, flags=flags)
+        res = tm.tilemix_attention_fwd(p, qd, kd, vd, None, None, None, None, None)
+        assert tm.tilemix_read_status(res["workspace"])[0] == 0
+        outs.append(res["out"])
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
