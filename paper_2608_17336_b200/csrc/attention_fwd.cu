@@ -11,9 +11,10 @@
 //   warps 9, 10 MMA issuers      (one thread per query tile): tcgen05.mma kind::f16 or kind::i8 for
 //                                S = Q K^T per the routing bit, then kind::f16 for O += P V with P read
 //                                from tensor memory; warp 9 also owns the TMEM allocation
-//   warp  11    idle, or -- in the on-the-fly operand mode -- the on-chip quantiser: it makes the INT8
-//                                copies of the query tiles and of the key tiles routed to INT8 in
-//                                shared memory from the FP16 tiles (no INT8 operands in global memory)
+//   warp  11    idle
+//   warps 12-15 only in the on-the-fly operand mode: the on-chip quantiser, which makes the INT8 copies of
+//                                the query tiles and of the key tiles routed to INT8 in shared memory
+//                                from the FP16 tiles (no INT8 operands in global memory)
 // Tensor memory: S_A | S_B | O_A | O_B (FP32 / INT32 accumulators); the FP16 probabilities P
 // overwrite the first half of their S columns.  The two groups alternate: while group A turns
 // S_A into P_A on the ALUs, the tensor pipe runs PV_B and the next QK_B, and vice versa.
@@ -35,9 +36,14 @@ namespace {
 constexpr int kWarpsPerGroup = 4;
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr int kQuantWarp = 11;          // on-chip quantiser of the on-the-fly mode (idle otherwise)
 constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
 constexpr int kRegsSoftmax = 216, kRegsOther = 72;   // setmaxnreg split: 2*128*216 + 128*72 = 64512 of the 65536 registers
+// On-the-fly operand mode: a fourth warpgroup, the on-chip quantiser (32 rows of a tile per warp).  512 threads
+// start with 128 registers each; 2*128*200 + 2*128*56 = 65536 stays inside that allotment.
+constexpr int kQuantWarp0 = 12, kQuantWarps = 4;
+constexpr int kThreadsOtf = 512;
+constexpr int kRegsSoftmaxOtf = 200, kRegsOtherOtf = 56;
+constexpr uint32_t kQuantBar = 9;         // named barrier of the quantiser warps
 constexpr int kRing = 8;
 constexpr int kBundles = 4;        // operand bundles in flight at most (each has a "landed" and a "consumed" barrier)
 constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
@@ -184,7 +190,7 @@ struct Ring {
 // and no scales in global memory; a quantiser warp makes them in shared memory from the FP16 tiles, for
 // the key tiles some query tile of the CTA routes to INT8 only.
 template <int D, int T, bool VL, bool OTF>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(OTF ? kThreadsOtf : kThreads, 1)
 attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                  const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16,
                  const __grid_constant__ CUtensorMap tm_q8, const __grid_constant__ CUtensorMap tm_k8) {
@@ -268,14 +274,14 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         ptx::mbar_init(bar_q(0), 1);
         ptx::mbar_init(bar_q(1), 1);
         for (int i = 0; i < kBundles; ++i) {
-            // on-the-fly mode: a second arrival, by the quantiser (after it made the bundle's INT8 tile, if
-            // there is one to make)
-            ptx::mbar_init(bar_full(i), OTF ? 2 : 1);
+            // on-the-fly mode: one more arrival per quantiser warp (after it made its rows of the bundle's INT8
+            // tile, if there is one to make)
+            ptx::mbar_init(bar_full(i), OTF ? 1 + kQuantWarps : 1);
             ptx::mbar_init(bar_empty(i), hasB ? 2 : 1);   // one arrival per MMA issuer
             ptx::mbar_init(bar_raw(i), 2);                // K16 bytes expected + "INT8 chunk claimed"
         }
-        ptx::mbar_init(bar_q8(0), 1);
-        ptx::mbar_init(bar_q8(1), 1);
+        ptx::mbar_init(bar_q8(0), kQuantWarps);
+        ptx::mbar_init(bar_q8(1), kQuantWarps);
         for (int t = 0; t < 2; ++t) {
             for (int h = 0; h < 2; ++h) {
                 ptx::mbar_init(bar_s(t, h), 1);
@@ -291,7 +297,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // Schedule table, one 4-bit entry per key tile j (Sec. 4.2 lookup done once per CTA):
     //   bit0 / bit1: tile A / tile B takes the INT8 route at key tile j  (R = (b >> floor(j/G)) & 1)
     //   bit2 / bit3: the FP16 / the INT8 copy of K_j has to be staged
-    for (int i = threadIdx.x; i * 8 < nkv; i += kThreads) {
+    for (int i = threadIdx.x; i * 8 < nkv; i += blockDim.x) {
         uint32_t packed = 0u;
         for (int jj = 0; jj < 8; ++jj) {
             const int j = i * 8 + jj;
@@ -322,61 +328,81 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const uint32_t tmem_base = misc[0];
     auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
-    if (OTF && warp == kQuantWarp) {
+    if (OTF && warp >= kQuantWarp0) {
         // ================================================================ on-chip quantiser (on-the-fly mode)
-        // One warp makes the INT8 copies the tensor pipe reads: of the two query tiles once, then of every
-        // key tile some query tile of the CTA routes to INT8.  A tile is 128 rows = one quantisation block
-        // (App. C): delta = max|x| / 127 over the tile, codes by the quantiser's own arithmetic.  Source and
+        // Four warps make the INT8 copies the tensor pipe reads: of a query tile before the first key tile it
+        // routes to INT8, then of every key tile some query tile of the CTA routes to INT8.  A tile is 128
+        // rows = one quantisation block (App. C): delta = max|x| / 127 over the tile, codes by the quantiser's
+        // own arithmetic; each warp takes 32 rows, the four partial maxima meet in shared memory.  Source and
         // destination are the shared-memory images TMA would have written: FP16 tiles as D/64 slabs of
         // 128-byte rows, INT8 tiles as 128-byte rows, both with the 128-byte swizzle (16-byte chunk c of row r
         // sits at chunk c ^ (r & 7)).
-        ptx::setmaxnreg_dec<kRegsOther>();
+        ptx::setmaxnreg_dec<OTF ? kRegsOtherOtf : kRegsOther>();
         static_assert(!OTF || (D == 128 && T == 128), "the on-chip quantiser handles 128 x 128 tiles");
+        const int cw = warp - kQuantWarp0;
+        volatile uint32_t* xch = misc + 2;   // partial maxima of the four warps: words 2, 3, 14, 15 of misc
+        auto xch_slot = [&](int w) -> volatile uint32_t& { return xch[w < 2 ? w : w + 10]; };
+        // `ok` turns false when a bounded wait ran out or the CTA is aborting; a warp then skips the work but
+        // keeps meeting the others at the named barrier (every warp runs the same number of tiles).
         bool ok = true;
         auto quantise_tile = [&](uint32_t src_off, uint32_t dst_off) -> float {
             const uint8_t* src = smem + src_off;
             uint8_t* dst = smem + dst_off;
-            constexpr int kVec = C::kHalves * 128 * 8;   // 16-byte vectors (8 elements) of the FP16 tile
+            constexpr int kRowsW = 128 / kQuantWarps, kVecW = kRowsW * 8;   // rows / 16-byte vectors per warp and slab
             uint32_t amax2 = 0u;
-            for (int i0 = lane; i0 < kVec; i0 += 32 * 8) {   // eight loads in flight per lane
-                uint4 v[8];
+            if (ok) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = *reinterpret_cast<const uint4*>(src + (i0 + 32 * u) * 16);
+                for (int sl = 0; sl < C::kHalves; ++sl) {
+                    uint4 v[kVecW / 32];   // eight loads in flight per lane
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    amax2 = umax2(amax2, umax2(umax2(habs2_bits(v[u].x), habs2_bits(v[u].y)),
-                                               umax2(habs2_bits(v[u].z), habs2_bits(v[u].w))));
+                    for (int u = 0; u < kVecW / 32; ++u)
+                        v[u] = *reinterpret_cast<const uint4*>(src + (sl * 1024 + cw * kVecW + lane + 32 * u) * 16);
+#pragma unroll
+                    for (int u = 0; u < kVecW / 32; ++u)
+                        amax2 = umax2(amax2, umax2(umax2(habs2_bits(v[u].x), habs2_bits(v[u].y)),
+                                                   umax2(habs2_bits(v[u].z), habs2_bits(v[u].w))));
+                }
             }
             uint32_t amax = max(amax2 & 0xffffu, amax2 >> 16);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0) xch_slot(cw) = amax;
+            ptx::bar_sync_named(kQuantBar, kQuantWarps * 32);
+            amax = max(max(xch_slot(0), xch_slot(1)), max(xch_slot(2), xch_slot(3)));
+            ptx::bar_sync_named(kQuantBar, kQuantWarps * 32);   // all have read: the slots may be written again
             const float amax_f = __half2float(__ushort_as_half(static_cast<unsigned short>(amax)));
             const float delta = __fdiv_rn(amax_f, 127.0f);
+            if (!ok) return delta;
             if (amax == 0u) {   // zero block: delta = 0, every code 0
-                for (int i = lane; i < 128 * D / 16; i += 32)
-                    *reinterpret_cast<uint4*>(dst + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+                for (int i = lane; i < kRowsW * D / 16; i += 32)
+                    *reinterpret_cast<uint4*>(dst + cw * kRowsW * 128 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
                 return delta;
             }
             const float rdelta = __frcp_rn(delta);
-            for (int i0 = lane; i0 < kVec; i0 += 32 * 4) {   // four vectors in flight per lane
-                uint4 v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const uint4*>(src + (i0 + 32 * u) * 16);
-                uint2 qv[4];
+            for (int sl = 0; sl < C::kHalves; ++sl) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) qv[u] = quant8_div(v[u], delta, rdelta);
+                for (int u0 = 0; u0 < kVecW / 32; u0 += 4) {   // four vectors in flight per lane
+                    uint4 v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + 32 * u;
-                    const int slab = i >> 10, r = (i >> 3) & 127, cl = (i & 7) ^ (r & 7);   // logical chunk of the slab
-                    // elements 64 slab + 8 cl .. + 7 of row r: byte column 64 slab + 8 cl of the INT8 row
-                    const int c16 = slab * 4 + (cl >> 1);
-                    *reinterpret_cast<uint2*>(dst + r * 128 + ((c16 ^ (r & 7)) << 4) + (cl & 1) * 8) = qv[u];
+                    for (int u = 0; u < 4; ++u)
+                        v[u] = *reinterpret_cast<const uint4*>(src + (sl * 1024 + cw * kVecW + lane + 32 * (u0 + u)) * 16);
+                    uint2 qv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) qv[u] = quant8_div(v[u], delta, rdelta);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = cw * kVecW + lane + 32 * (u0 + u);          // vector of the slab
+                        const int r = i >> 3, cl = (i & 7) ^ (r & 7);             // row, logical chunk of the slab
+                        // elements 64 sl + 8 cl .. + 7 of row r: byte column 64 sl + 8 cl of the INT8 row
+                        const int c16 = sl * 4 + (cl >> 1);
+                        *reinterpret_cast<uint2*>(dst + r * 128 + ((c16 ^ (r & 7)) << 4) + (cl & 1) * 8) = qv[u];
+                    }
                 }
             }
             return delta;
         };
-        // hand-over to the async proxy (the tensor pipe reads shared memory through it), then one arrival
+        // hand-over to the async proxy (the tensor pipe reads shared memory through it), then one arrival per warp
         auto publish = [&](uint32_t bar) {
             ptx::fence_proxy_async_smem();
             __syncwarp();
@@ -384,11 +410,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         };
         // The quantiser arrives on the "landed" barrier of EVERY bundle, with or without an INT8 tile to
         // make, so that the issuers (and with them the producer) can never run more than kBundles bundles
-        // ahead of it and the phase it waits for is unambiguous.  A query tile is quantised just before the
-        // first key tile it routes to INT8.
+        // ahead of it and the phase it waits for is unambiguous.
         Ring ring;   // the producer's sequence of chunks
         uint32_t q8_made = 0u;
-        for (int n = 0; n < nkv && ok; ++n) {
+        for (int n = 0; n < nkv; ++n) {
             const uint32_t e = sched(n);
             uint32_t s16 = 0, s8 = 0;
             if (n >= 1) ring.take(C::kHalves);
@@ -396,29 +421,26 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if (e & 8u) s8 = ring.take(1);
             for (int t = 0; t < 2; ++t) {
                 if (!((e >> t) & 1u) || ((q8_made >> t) & 1u)) continue;
-                ok = wait_bar(cx, bar_q(t), 0, kRoleQuant, t, kBarQ);
+                if (ok) ok = wait_bar(cx, bar_q(t), 0, kRoleQuant, t, kBarQ);
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
                 const float dq = quantise_tile(C::kOffQ16 + t * C::kQ16Tile, C::kOffQ8 + t * C::kQ8Tile);
-                if (lane == 0) otf_dq[t] = dq;
+                if (cw == 0 && lane == 0) otf_dq[t] = dq;
                 publish(bar_q8(t));
                 q8_made |= 1u << t;
             }
-            if (!ok) break;
-            ok = wait_bar(cx, bar_raw(n % kBundles), (n / kBundles) & 1, kRoleQuant, n, kBarRaw);
+            if (ok) ok = wait_bar(cx, bar_raw(n % kBundles), (n / kBundles) & 1, kRoleQuant, n, kBarRaw);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
             if (e & 8u) {
                 const float dk = quantise_tile(C::kOffRing + s16 * C::kChunk, C::kOffRing + s8 * C::kChunk);
-                if (lane == 0) otf_dk[n % (2 * kBundles)] = dk;
+                if (cw == 0 && lane == 0) otf_dk[n % (2 * kBundles)] = dk;
             }
             publish(bar_full(n % kBundles));
         }
     } else if (warp >= kMmaWarp + 2 || (warp == kMmaWarp + 1 && !hasB)) {
-        ptx::setmaxnreg_dec<kRegsOther>();   // idle warps of the third warpgroup
+        ptx::setmaxnreg_dec<OTF ? kRegsOtherOtf : kRegsOther>();   // idle warps of the third warpgroup
     } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer
-        ptx::setmaxnreg_dec<kRegsOther>();
+        ptx::setmaxnreg_dec<OTF ? kRegsOtherOtf : kRegsOther>();
         if (lane == 0) {
             ptx::tma_prefetch_desc(&tm_q16);
             ptx::tma_prefetch_desc(&tm_k16);
@@ -472,7 +494,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (bytes != 0u) ptx::mbar_arrive_expect_tx(bar, bytes);
                 else ptx::mbar_arrive(bar);
                 if (OTF) {
-                    if (n == nkv) ptx::mbar_arrive(bar);   // the last bundle (V only) is not the quantiser's
+                    if (n == nkv)                          // the last bundle (V only) is not the quantiser's
+                        for (int w = 0; w < kQuantWarps; ++w) ptx::mbar_arrive(bar);
                     if (n < nkv) {
                         if (raw_bytes != 0u) ptx::mbar_arrive_expect_tx(bar_raw(n % kBundles), raw_bytes);
                         else ptx::mbar_arrive(bar_raw(n % kBundles));
@@ -521,7 +544,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         // ================================================================ MMA issuers
         // One issuing thread per query tile (warp kMmaWarp: tile A, the next warp: tile B).  Both walk
         // the same sequence of ring items; an item goes back to the producer when both have committed it.
-        ptx::setmaxnreg_dec<kRegsOther>();
+        ptx::setmaxnreg_dec<OTF ? kRegsOtherOtf : kRegsOther>();
         if (lane == 0) {
             const int t = warp - kMmaWarp;
             const int m_t = t ? kB : kA;       // last key tile of this issuer's query tile
@@ -644,7 +667,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         }
     } else {
         // ================================================================ softmax groups
-        ptx::setmaxnreg_inc<kRegsSoftmax>();
+        ptx::setmaxnreg_inc<OTF ? kRegsSoftmaxOtf : kRegsSoftmax>();
         const int t = warp / kWarpsPerGroup;
         const int m_t = t ? mB : mA;           // query-tile row
         const int k_t = t ? kB : kA;           // its diagonal key tile
@@ -1020,7 +1043,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
                             : static_cast<int64_t>(g.B) * g.Hq * ((g.T_m + 1) / 2);
     if (ctas == 0) return TILEMIX_OK;   // only zero-length sequences
     if (ctas > 0x7fffffffLL) return static_cast<int>(cudaErrorInvalidConfiguration);
-    kernel<<<static_cast<unsigned>(ctas), kThreads, C::kSmemAlloc, stream>>>(prm, tq, tk, tv, tq8, tk8);
+    kernel<<<static_cast<unsigned>(ctas), otf ? kThreadsOtf : kThreads, C::kSmemAlloc, stream>>>(prm, tq, tk, tv, tq8, tk8);
     g_launch_count.fetch_add(1);
     return static_cast<int>(cudaGetLastError());
 }

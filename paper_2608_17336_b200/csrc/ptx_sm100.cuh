@@ -239,5 +239,10 @@ __device__ __forceinline__ void tmem_wait_st() {
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// Named barrier (ids 1..15; id 0 is __syncthreads) among `threads` threads (a multiple of 32).
+__device__ __forceinline__ void bar_sync_named(uint32_t id, uint32_t threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 }  // namespace ptx
 }  // namespace tilemix
