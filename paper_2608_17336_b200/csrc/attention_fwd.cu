@@ -200,11 +200,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     const uint32_t sbase = ptx::smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // An earlier CTA of this launch already failed: do nothing (decided once per CTA).
+    // An earlier CTA of this launch already failed: do nothing (decided once per CTA; the status word is read
+    // here and looked at behind the set-up barrier, so that its latency hides behind the set-up).
     __shared__ int s_skip;
-    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int*>(prm.status);
-    __syncthreads();
-    if (s_skip != 0) return;
+    int skip_word = 0;
+    if (threadIdx.x == 0) skip_word = *reinterpret_cast<volatile int*>(prm.status);
 
 #ifdef TILEMIX_PHASE_TIMERS
     const long long cta_c0 = clock64();
@@ -293,6 +293,21 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         ptx::mbar_init(bar_drain, hasB ? 2 : 1);
         misc[1] = 0;
         ptx::fence_mbar_init();
+        s_skip = skip_word;
+        // The query tiles do not depend on the schedule table: their copies start here, ahead of the set-up
+        // barrier, and land while the table is being built.
+        if (skip_word == 0) {
+            for (int t = 0; t < (hasB ? 2 : 1); ++t) {
+                const int m = t ? mB : mA;
+                const uint32_t bytes = C::kQ16Tile + ((prm.has_int8 && !OTF) ? C::kQ8Tile : 0);
+                ptx::mbar_arrive_expect_tx(bar_q(t), bytes);
+                for (int c = 0; c < C::kHalves; ++c)
+                    ptx::tma_load_4d(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, &tm_q16,
+                                     bar_q(t), c * 64, tok0 + m * T, hq, b);
+                if (prm.has_int8 && !OTF)
+                    ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
+            }
+        }
     }
     // Schedule table, one 4-bit entry per key tile j (Sec. 4.2 lookup done once per CTA):
     //   bit0 / bit1: tile A / tile B takes the INT8 route at key tile j  (R = (b >> floor(j/G)) & 1)
@@ -326,6 +341,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc[0];
+    if (s_skip != 0) {   // nothing is in flight (no copy was started): give the tensor memory back and leave
+        if (warp == kMmaWarp) ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+        return;
+    }
     auto sched = [&](int j) -> uint32_t { return (sched_s[j >> 3] >> ((j & 7) * 4)) & 15u; };
 
     if (OTF && warp >= kQuantWarp0) {
@@ -448,16 +467,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if (prm.has_int8 && !OTF) {
                 ptx::tma_prefetch_desc(&tm_q8);
                 ptx::tma_prefetch_desc(&tm_k8);
-            }
-            for (int t = 0; t < (hasB ? 2 : 1); ++t) {
-                const int m = t ? mB : mA;
-                const uint32_t bytes = C::kQ16Tile + ((prm.has_int8 && !OTF) ? C::kQ8Tile : 0);
-                ptx::mbar_arrive_expect_tx(bar_q(t), bytes);
-                for (int c = 0; c < C::kHalves; ++c)
-                    ptx::tma_load_4d(sbase + C::kOffQ16 + t * C::kQ16Tile + c * C::kQ16Slab, &tm_q16,
-                                     bar_q(t), c * 64, tok0 + m * T, hq, b);
-                if (prm.has_int8 && !OTF)
-                    ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
             }
             // Chunks are taken from the ring in the order K16_j?, K8_j?, V_j (j = 0, 1, ...), the same
             // order in which the issuers count them.  A chunk may be refilled once the bundle that used it
