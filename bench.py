@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
 # profiles/attention_kernel_cfg3_long32k.md (8-head capture: 320.6 MB, traffic scales with the head count).
-NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 320.6e6 / 8}
+NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 321.1e6 / 8}
 
 
 def effective_flops(w: synth.Workload) -> float:
