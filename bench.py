@@ -31,7 +31,7 @@ METRIC = "effective causal-attention TFLOP/s at 1 B200 vs INT8 fraction; % of mi
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
-# profiles/attention_kernel_cfg3_long32k.md (8-head capture: 320.6 MB, traffic scales with the head count).
+# profiles/attention_kernel_cfg3_long32k.md (8-head capture: 321.1 MB, traffic scales with the head count).
 NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 321.1e6 / 8}
 
 
