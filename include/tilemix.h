@@ -269,15 +269,16 @@ typedef struct tilemix_decode {
     float softmax_scale;   /* <= 0 means 1/sqrt(head_dim)                                   */
 } tilemix_decode_t;
 
-/* Bytes of `workspace` for tilemix_decode_int8kv: the partial results of the splits
- * (0 on an invalid problem). */
+/* Bytes of `workspace` for tilemix_decode_int8kv: the status record, the clamped copy of the cache lengths
+ * and the partial results of the splits (0 on an invalid problem). */
 size_t tilemix_decode_workspace_size(const tilemix_decode_t* p);
 /*   q_f16      FP16 [B, Hq, d]
  *   k_f16      FP16 [B, Hk, max_len, d]   (may be NULL if every legal group is INT8-routed:
  *                                          a 0 bit then reads NULL -- the caller's contract)
  *   k_i8, v_i8 INT8 [B, Hk, max_len, d];  k_scale, v_scale FP32 [B, Hk, ceil(max_len/tile_n)]
  *   mask_words uint32 [nb, Hk, W], W = ceil(ceil(max_len/(G*tile_n))/32); NULL = all FP16
- *   cache_len  int32 [B] on the DEVICE, 0 <= cache_len[b] <= max_len; a sequence of length 0
+ *   cache_len  int32 [B] on the DEVICE, 0 <= cache_len[b] <= max_len (values outside are clamped to that
+ *              range by the kernel); a sequence of length 0
  *              gets an all-zero output row and lse = -inf
  *   out_f16    FP16 [B, Hq, d];  lse nullable FP32 [B, Hq]
  *   q_i8_out / q_scale_out  nullable INT8 [B, Hq, d] / FP32 [B, Hq]: the quantised query the

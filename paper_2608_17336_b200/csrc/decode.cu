@@ -98,7 +98,8 @@ decode_kernel(const DecodeParams prm) {
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int len = prm.cache_len[b];
+    // (lengths live on the device and cannot be checked by the host: out-of-range values are clamped)
+    const int len = prm.cache_len[b];   // the clamped copy decode_prepare_kernel made
     const int n_tiles = (len + T - 1) / T;
     const int per_split = (n_tiles + prm.n_splits - 1) / prm.n_splits;
     const int t0 = split * per_split, t1 = min(n_tiles, t0 + per_split);
@@ -449,8 +450,6 @@ int launch_cfg(const DecodeParams& prm, __half* out, float* lse, cudaStream_t st
     auto kernel = prm.k16 != nullptr ? decode_kernel<D, R, T, true> : decode_kernel<D, R, T, false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRing);
     if (e != cudaSuccess) return static_cast<int>(e);
-    e = cudaMemsetAsync(prm.status, 0, 16, stream);
-    if (e != cudaSuccess) return static_cast<int>(e);
     kernel<<<grid, kDecodeThreads, kRing, stream>>>(prm);
     g_launch_count.fetch_add(1);
     e = cudaGetLastError();
@@ -472,6 +471,17 @@ int launch_r(int R, const DecodeParams& prm, __half* out, float* lse, cudaStream
 }
 
 constexpr size_t kDecodeStatusBytes = 256;   // status record of the bounded waits
+
+// Before the step: clears the status record and copies the cache lengths, clamped to [0, max_len], into the
+// workspace (they live on the device, so the host cannot check them; the step itself reads the copy).
+__global__ void decode_prepare_kernel(const int32_t* __restrict__ cache_len, int B, int max_len, int* status,
+                                      int32_t* __restrict__ len_out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < 4) status[i] = 0;
+    if (i < B) len_out[i] = min(max(cache_len[i], 0), max_len);
+}
+
+size_t decode_len_bytes(int B) { return (static_cast<size_t>(B) * sizeof(int32_t) + 255) / 256 * 256; }
 
 struct DecodeGeometry {
     int n_blk, T_mask, W, n_splits;
@@ -521,7 +531,7 @@ extern "C" {
 size_t tilemix_decode_workspace_size(const tilemix_decode_t* p) {
     DecodeGeometry g;
     if (resolve_decode(p, &g)) return 0;
-    return kDecodeStatusBytes + g.o_bytes + 2 * g.mz_bytes;
+    return kDecodeStatusBytes + decode_len_bytes(p->batch) + g.o_bytes + 2 * g.mz_bytes;
 }
 
 int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const void* k_f16, const int8_t* k_i8,
@@ -537,7 +547,7 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     if (!aligned16(q_f16) || !aligned16(k_i8) || !aligned16(v_i8) || !aligned16(out_f16) || !aligned16(workspace) ||
         (k_f16 && !aligned16(k_f16)))
         return TILEMIX_ERR_ALIGN;
-    if (workspace_bytes < kDecodeStatusBytes + g.o_bytes + 2 * g.mz_bytes) return TILEMIX_ERR_WORKSPACE;
+    if (workspace_bytes < kDecodeStatusBytes + decode_len_bytes(p->batch) + g.o_bytes + 2 * g.mz_bytes) return TILEMIX_ERR_WORKSPACE;
     DecodeParams prm{};
     prm.B = p->batch; prm.Hq = p->heads_q; prm.Hk = p->heads_kv; prm.max_len = p->max_len; prm.G = p->group;
     prm.nb = p->mask_batch; prm.W = g.W; prm.n_splits = g.n_splits; prm.n_blk = g.n_blk;
@@ -547,9 +557,11 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     prm.q = static_cast<const __half*>(q_f16);
     prm.k16 = static_cast<const __half*>(k_f16);
     prm.k8 = k_i8; prm.k_scale = k_scale; prm.v8 = v_i8; prm.v_scale = v_scale;
-    prm.words = mask_words; prm.cache_len = cache_len;
+    prm.words = mask_words;
     prm.status = static_cast<int*>(workspace);
-    uint8_t* ws = static_cast<uint8_t*>(workspace) + kDecodeStatusBytes;
+    int32_t* len_ws = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kDecodeStatusBytes);
+    prm.cache_len = len_ws;
+    uint8_t* ws = static_cast<uint8_t*>(workspace) + kDecodeStatusBytes + decode_len_bytes(p->batch);
     prm.o_part = reinterpret_cast<float*>(ws);
     prm.m_part = reinterpret_cast<float*>(ws + g.o_bytes);
     prm.z_part = reinterpret_cast<float*>(ws + g.o_bytes + g.mz_bytes);
@@ -557,6 +569,11 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int R = p->heads_q / p->heads_kv;
     __half* out = static_cast<__half*>(out_f16);
+    const int prep_threads = p->batch > 4 ? p->batch : 4;
+    decode_prepare_kernel<<<(prep_threads + 255) / 256, 256, 0, s>>>(cache_len, p->batch, p->max_len, prm.status, len_ws);
+    g_launch_count.fetch_add(1);
+    cudaError_t pe = cudaGetLastError();
+    if (pe != cudaSuccess) return static_cast<int>(pe);
     // keys are streamed and processed one routing tile at a time (64-key chunks with a deeper ring
     // were slower: the per-chunk barriers cost more than the extra bytes in flight gain)
     if (p->head_dim == 128 && p->tile_n == 128) return launch_r<128, kChunk>(R, prm, out, lse, s);

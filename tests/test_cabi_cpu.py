@@ -191,10 +191,11 @@ def test_varlen_host_side_validation(lib):
 def test_decode_host_side_validation(lib):
     ok = b.decode_problem(8, 32, 8, 128, 32768, 128, 4)
     size = lib.tilemix_decode_workspace_size(ctypes.byref(ok))
-    # 256-byte status area + partial outputs and two float arrays per (batch, query head, split)
-    splits = (size - 256) // (8 * 32 * (128 * 4 + 8))
-    assert splits >= 1 and size == 256 + 8 * 32 * splits * (128 * 4 + 8)
-    assert b.tilemix_decode_workspace_size(b.decode_problem(1, 4, 1, 64, 64, 64, n_splits=7)) == 256 + 1024 + 2 * 256
+    # 256-byte status area + the clamped lengths (a 256-byte area for up to 64 sequences) + partial outputs and
+    # two float arrays per (batch, query head, split)
+    splits = (size - 512) // (8 * 32 * (128 * 4 + 8))
+    assert splits >= 1 and size == 512 + 8 * 32 * splits * (128 * 4 + 8)
+    assert b.tilemix_decode_workspace_size(b.decode_problem(1, 4, 1, 64, 64, 64, n_splits=7)) == 256 + 256 + 1024 + 2 * 256
     for bad in (b.decode_problem(0, 32, 8, 128, 1024, 128), b.decode_problem(1, 6, 4, 128, 1024, 128),
                 b.decode_problem(1, 4, 4, 128, 0, 128), b.decode_problem(2, 4, 4, 128, 1024, 128, mask_batch=3)):
         assert lib.tilemix_decode_workspace_size(ctypes.byref(bad)) == 0

@@ -128,3 +128,12 @@ def test_decode_random_shapes(seed):
     lens = rng.integers(0, L + 1, B).tolist()
     q, k, v, route, lens = _case(B, Hk * rep, Hk, L, d, tile, G, seed=seed, lens=lens, f8=float(rng.random()))
     _check(q, k, v, route, lens, tile, G, n_splits=int(rng.integers(0, 6)))
+
+
+def test_decode_out_of_range_lengths_are_clamped():
+    """cache_len lives on the device; a value above max_len acts as max_len, a negative one as 0."""
+    q, k, v, route, _ = _case(3, 4, 2, 300, 128, 128, 1, seed=41, lens=[0, 0, 0])
+    good, _ = _gpu(q, k, v, route, np.asarray([300, 0, 123], np.int32), 128, 1)
+    bad, _ = _gpu(q, k, v, route, np.asarray([100000, -5, 123], np.int32), 128, 1)
+    assert torch.equal(good["out"].view(torch.int16), bad["out"].view(torch.int16))
+    assert torch.equal(good["lse"], bad["lse"])
