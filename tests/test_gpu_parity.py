@@ -342,3 +342,48 @@ def test_prefill_host_equals_device_path(B, Hq, Hk, nb):
                                      torch.from_numpy(route).pin_memory(), out, arena, pin_diagonal=True)
         torch.cuda.current_stream().synchronize()
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103])
+def test_attention_random_shapes(seed):
+    """Random dense cases -- batch, GQA ratio, length (ragged), tile, group, INT8 share, pin, value recipe, shared or
+    per-batch mask -- through the whole path: quantiser and packer bit-exact, sampled rows against the oracle."""
+    from paper_2608_17336_b200 import binding as tm
+    rng = np.random.default_rng(seed)
+    dev = torch.device("cuda:0")
+    for it in range(8):
+        tile = int(rng.choice([64, 128]))
+        hk = int(rng.choice([1, 2]))
+        hq = hk * int(rng.choice([1, 2, 4]))
+        B = int(rng.choice([1, 2, 3]))
+        L = int(rng.integers(1, 9 * tile))
+        G = int(rng.choice([1, 2, 3, 5]))
+        f8 = float(rng.choice([0.0, 0.3, 0.5, 0.8, 1.0]))
+        pin = bool(rng.integers(0, 2))
+        mb = int(rng.choice([1, B]))
+        w = synth.Workload("rnd", B, hq, L, tile, tile, G, seed=seed * 100 + it,
+                           values=str(rng.choice(["normal", "outlier_channels", "student_t_k"])),
+                           routing=str(rng.choice(["bernoulli", "row_exact"])), int8_fraction=f8, pin_diagonal=pin,
+                           mask_batch=mb)
+        q, k, v = synth.make_qkv(w)
+        k, v = k[:, :hk].contiguous(), v[:, :hk].contiguous()
+        route = np.ascontiguousarray(synth.make_route(w)[:, :hk])
+        qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+        p = tm.problem(B, hq, hk, L, tile, tile, tile, G, mask_batch=mb)
+        q8, k8, qs, ks = tm.tilemix_quantize_qk(p, qd, kd)
+        words, _ = tm.tilemix_pack_routing_mask(p, torch.from_numpy(route).to(dev), pin)
+        res = tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words)
+        code, rec = tm.tilemix_read_status(res["workspace"])
+        assert code == 0, rec
+        po = oracle.Problem(B, hq, hk, L, tile, tile, tile, G, mask_batch=mb)
+        qb, kb, vb = H.np_bits(q), H.np_bits(k), H.np_bits(v)
+        q8o, qso = oracle.quantize(qb, tile)
+        k8o, kso = oracle.quantize(kb, tile)
+        assert np.array_equal(q8.cpu().numpy(), q8o) and np.array_equal(k8.cpu().numpy(), k8o)
+        wo, _ = oracle.pack(po, route, pin)
+        assert np.array_equal(words.cpu().numpy().view(np.uint32), wo)
+        rows = [(b, h, int(i)) for b in range(B) for h in range(hq)
+                for i in rng.choice(L, size=min(L, 8), replace=False)]
+        ref, _, _ = oracle.attention_rows(po, qb, kb, vb, q8o, k8o, qso, kso, wo, rows)
+        got = np.stack([res["out"][b, h, i].float().cpu().numpy() for b, h, i in rows]).astype(np.float64)
+        assert (np.abs(got - ref) <= H.ATOL * np.maximum(1.0, np.abs(ref))).all(), (it, B, hq, hk, L, tile, G, f8, pin)
