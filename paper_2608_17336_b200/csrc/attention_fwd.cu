@@ -44,6 +44,7 @@ constexpr int kQuantWarp0 = 12, kQuantWarps = 4;
 constexpr int kThreadsOtf = 512;
 constexpr int kRegsSoftmaxOtf = 200, kRegsOtherOtf = 56;
 constexpr uint32_t kQuantBar = 9;         // named barrier of the quantiser warps
+constexpr int kMaxHeadGroup = 8;   // (batch, head) rows whose CTAs are interleaved in the grid order, at most
 constexpr int kRing = 8;
 constexpr int kBundles = 4;        // operand bundles in flight at most (each has a "landed" and a "consumed" barrier)
 constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
@@ -99,6 +100,7 @@ struct Cfg {
 struct Params {
     int B, Hq, Hk, L, G, T_m, W, nb;
     int kv_off, mask_T_m, ks_blocks;   // chunked prefill: see Geometry (0, T_m, T_m for a plain prefill)
+    int head_group;               // (batch, head) rows interleaved in the grid order (>= 1)
     int has_int8;                 // INT8 operands present
     float scale_log2;             // softmax scale * log2(e)
     const float* q_scale;         // [B,Hq,T_m]; variable-length batch: [sum T_m, Hq]
@@ -214,16 +216,29 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // tok0 / len: first token and length of the sequence; row0: its first row among the mask rows
     // and scale blocks; m, n below count tiles inside the sequence.
     int b, hq, pr, seq, tok0 = 0, len = prm.L, row0 = VL ? 0 : prm.kv_off, n_rows = prm.T_m;
+    // Order of the grid: (batch, head) rows in groups of head_group; inside a group the longest work items
+    // first, and the heads of the group side by side for each item.  The host sizes the group so that its
+    // K/V fits in L2 while its CTAs run; the grid then ends with the shortest items of the last group instead
+    // of with the long items of the last head, and the SMs finish close together.
+    const int kHeadGroup = prm.head_group;
     if constexpr (!VL) {
         const int n_pairs = (prm.T_m + 1) >> 1;
-        const int bh = blockIdx.x / n_pairs;
-        pr = n_pairs - 1 - (blockIdx.x - bh * n_pairs);   // longest rows first
+        const int n_bh = prm.B * prm.Hq;
+        const int grp = blockIdx.x / (kHeadGroup * n_pairs);
+        const int in_grp = blockIdx.x - grp * (kHeadGroup * n_pairs);
+        const int g_heads = min(kHeadGroup, n_bh - grp * kHeadGroup);    // the last group may be smaller
+        const int item = in_grp / g_heads;
+        const int bh = grp * kHeadGroup + (in_grp - item * g_heads);
+        pr = n_pairs - 1 - item;                            // longest rows first
         b = bh / prm.Hq;
         hq = bh - b * prm.Hq;
         seq = b;
     } else {
-        hq = blockIdx.x / prm.total_pairs;
-        const int item = blockIdx.x - hq * prm.total_pairs;
+        const int grp = blockIdx.x / (kHeadGroup * prm.total_pairs);
+        const int in_grp = blockIdx.x - grp * (kHeadGroup * prm.total_pairs);
+        const int g_heads = min(kHeadGroup, prm.Hq - grp * kHeadGroup);
+        const int item = in_grp / g_heads;                  // items are sorted by length on the host
+        hq = grp * kHeadGroup + (in_grp - item * g_heads);
         seq = prm.vl_item_seq[item];
         pr = prm.vl_item_pair[item];
         b = 0;
@@ -1024,6 +1039,15 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     Params prm{};
     prm.B = g.B; prm.Hq = g.Hq; prm.Hk = g.Hk; prm.L = g.L; prm.G = g.G; prm.T_m = g.T_m; prm.W = g.W;
     prm.kv_off = g.kv_off; prm.mask_T_m = g.mask_T_m; prm.ks_blocks = g.ks_blocks;
+    {
+        // heads per group: as many as keep the group's K and V (FP16; adjacent query heads of a GQA group share
+        // theirs) within 72 MB of the 126 MB L2
+        const int64_t kv_bytes = 2 * static_cast<int64_t>(g.Lk) * g.d * 2;
+        const int rep = g.Hq / g.Hk;
+        int hg = 1;
+        while (hg < kMaxHeadGroup && ceil_div(2 * hg, rep) * kv_bytes <= (72ll << 20)) hg *= 2;
+        prm.head_group = hg;
+    }
     prm.nb = g.nb;
     prm.has_int8 = has8 ? 1 : 0;
     prm.scale_log2 = g.scale * kLog2e;
