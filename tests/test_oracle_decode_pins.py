@@ -138,3 +138,42 @@ def test_int8_route_equals_fp16_route_when_quantisation_is_lossless():
     a, la = od.decode(*args, np.zeros_like(one), [L], tile, 1)
     b_, lb = od.decode(*args, one, [L], tile, 1)
     assert np.abs(a - b_).max() < 1e-12 and np.abs(la - lb).max() < 1e-12
+
+
+def test_per_batch_mask_rows_select_their_own_batch_entry():
+    """One mask row per batch entry (words [B, Hk, W]): entry b must equal the single-sequence step on
+    entry b's cache with entry b's row, and differ from what the other entry's row gives."""
+    B, Hq, Hk, L, d, tile, G = 2, 4, 2, 260, 32, 64, 1
+    c = _case(B, Hq, Hk, L, d, tile, G, seed=7, lens=[260, 131])
+    rng = np.random.default_rng(8)
+    route = (rng.random((B, Hk, -(-L // (tile * G)))) < 0.5).astype(np.uint8)
+    route[1] = 1 - route[0]
+    words = od.pack_row(route)
+    assert words.shape[0] == B
+    out, lse = _run(c, words=words)
+    for b in range(B):
+        sl = slice(b, b + 1)
+        one = od.decode(c["q16"][sl], c["k16"][sl], c["k8"][sl], c["ks"][sl], c["v8"][sl], c["vs"][sl],
+                        words[sl], c["lens"][sl], tile, G)
+        assert np.array_equal(one[0][0], out[b]) and np.array_equal(one[1][0], lse[b])
+        other = od.decode(c["q16"][sl], c["k16"][sl], c["k8"][sl], c["ks"][sl], c["v8"][sl], c["vs"][sl],
+                          words[1 - b:2 - b], c["lens"][sl], tile, G)
+        assert np.abs(other[0][0] - out[b]).max() > 1e-5
+    # and against explicit loops for one head of entry 1 (its own row, not entry 0's)
+    half = lambda bits: float(np.array(bits, np.uint16).view(np.float16))
+    b, hq, hk = 1, 3, 1
+    qv = [half(x) for x in c["q16"][b, hq]]
+    q8, dq = od.quantize_query(c["q16"])
+    s = []
+    for j in range(131):
+        g = j // (tile * G)
+        if route[b, hk, g]:
+            dot = sum(int(a) * int(x) for a, x in zip(q8[b, hq], c["k8"][b, hk, j]))
+            s.append(float(dq[b, hq]) * float(c["ks"][b, hk, j // tile]) * dot / math.sqrt(d))
+        else:
+            s.append(sum(a * half(x) for a, x in zip(qv, c["k16"][b, hk, j])) / math.sqrt(d))
+    m = max(s)
+    w = [math.exp(x - m) for x in s]
+    for e in range(0, d, 7):
+        o = sum(w[j] * float(c["vs"][b, hk, j // tile]) * int(c["v8"][b, hk, j, e]) for j in range(131)) / sum(w)
+        assert abs(o - out[b, hq, e]) < 1e-12

@@ -381,3 +381,57 @@ def test_memory_accounting_matches_printed_table():
     # an INT8 K tile of 128 x 128 is half the FP16 tile the on-the-fly mode reads
     assert 128 * 128 * 2 / 1024 == golden["on_the_fly_int8_qk_tile_read_kb"]
     assert 128 * 128 / 1024 == int(golden["quantize_once_int8_qk_tile_read_kb"])
+
+
+# --------------------------------------------------------------------------- per-batch routing maps
+
+def test_per_batch_masks_equal_single_batch_runs():
+    """App. B "Policy Construction and Sharing": a template may be shared over the batch (mask_batch = 1)
+    or not (mask_batch = B).  With one routing map per batch entry, entry b must be exactly the
+    single-batch problem on entry b's tensors with entry b's map -- packed words, counters and outputs --
+    and must differ from what entry b gives under the other entry's map (so a wrong batch index fails)."""
+    rng = np.random.default_rng(15)
+    B, Hq, Hk, L, d, tile, G = 2, 2, 1, 90, 16, 16, 2
+    p = Problem(B, Hq, Hk, L, d, tile, tile, G, mask_batch=B)
+    q, k, v = rand_qkv(rng, B, Hq, Hk, L, d, scale=1.5)
+    q8, k8, qs, ks = quantized(p, q, k)
+    route = (rng.random((B, Hk, p.T_m, p.T_mask)) < 0.5).astype(np.uint8)
+    route[1] = 1 - route[0]                               # the two maps disagree on every group
+    for pin in (False, True):
+        words, counts = oracle.pack(p, route, pin)
+        out, lse, _ = oracle.attention_full(p, q, k, v, q8, k8, qs, ks, words)
+        p1 = Problem(1, Hq, Hk, L, d, tile, tile, G, mask_batch=1)
+        for b in range(B):
+            sl = slice(b, b + 1)
+            w1, c1 = oracle.pack(p1, np.ascontiguousarray(route[sl]), pin)
+            assert (w1[0] == words[b]).all() and (c1[0] == counts[b]).all()
+            o1, l1, _ = oracle.attention_full(p1, *(np.ascontiguousarray(x[sl]) for x in (q, k, v, q8, k8, qs, ks)), w1)
+            assert (o1[0] == out[b]).all() and (l1[0] == lse[b]).all()
+            wrong, _ = oracle.pack(p1, np.ascontiguousarray(route[1 - b:2 - b]), pin)
+            o2, _, _ = oracle.attention_full(p1, *(np.ascontiguousarray(x[sl]) for x in (q, k, v, q8, k8, qs, ks)), wrong)
+            assert np.abs(o2[0] - out[b]).max() > 1e-4
+        # sampled rows take the same branch as the full evaluation
+        rows = [(b, h, i) for b in range(B) for h in range(Hq) for i in (0, 17, L - 1)]
+        o3, _, _ = oracle.attention_rows(p, q, k, v, q8, k8, qs, ks, words, rows)
+        for r, (b, h, i) in enumerate(rows):
+            assert (o3[r] == out[b, h, i]).all()
+
+
+def test_per_batch_masks_match_brute_force():
+    """The numpy brute force of the mixed route, with the element-level route map taken from route[b]."""
+    rng = np.random.default_rng(16)
+    B, Hq, Hk, L, d, tile, G = 3, 2, 2, 70, 16, 16, 1
+    p = Problem(B, Hq, Hk, L, d, tile, tile, G, mask_batch=B)
+    q, k, v = rand_qkv(rng, B, Hq, Hk, L, d, scale=1.5)
+    q8, k8, qs, ks = quantized(p, q, k)
+    route = (rng.random((B, Hk, p.T_m, p.T_mask)) < 0.5).astype(np.uint8)
+    words, _ = oracle.pack(p, route)
+    out, _, _ = oracle.attention_full(p, q, k, v, q8, k8, qs, ks, words)
+    ii, jj = np.meshgrid(np.arange(L), np.arange(L), indexing="ij")
+    p1 = Problem(1, Hq, Hk, L, d, tile, tile, G)
+    for b in range(B):
+        route_elem = route[b][:, ii // tile, (jj // tile) // G]
+        sl = slice(b, b + 1)
+        ref = brute_force_mixed(p1, q[sl], k[sl], v[sl], q8[sl], k8[sl], qs[sl], ks[sl], route_elem, 1 / np.sqrt(d))
+        assert np.abs(out[b] - ref[0]).max() < 1e-12
+    assert np.abs(out[0] - out[1]).max() > 1e-4
