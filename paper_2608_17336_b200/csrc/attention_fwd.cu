@@ -2,22 +2,22 @@
 // Sec. 3.1 online softmax, App. C score formulas).
 //
 // One CTA owns two adjacent query tiles (A = 2p, B = 2p+1) of one (batch, query head) and
-// streams the key/value tiles 0..B once for both.  Warp roles:
-//   warps 0-3   softmax group A  (one thread per query row of tile A)
-//   warps 4-7   softmax group B
-//   warp  8     TMA producer     (one thread): Q16/Q8 once, then per key tile the K operand(s)
-//                                the routing bits ask for (FP16 and/or INT8) and V, into a
-//                                ring of equally sized shared-memory chunks
-//   warps 9, 10 MMA issuers      (one thread per query tile): tcgen05.mma kind::f16 or kind::i8 for
-//                                S = Q K^T per the routing bit, then kind::f16 for O += P V with P read
-//                                from tensor memory; warp 9 also owns the TMEM allocation
-//   warp  11    idle
-//   warps 12-15 only in the on-the-fly operand mode: the on-chip quantiser, which makes the INT8 copies of
-//                                the query tiles and of the key tiles routed to INT8 in shared memory
-//                                from the FP16 tiles (no INT8 operands in global memory)
-// Tensor memory: S_A | S_B | O_A | O_B (FP32 / INT32 accumulators); the FP16 probabilities P
-// overwrite the first half of their S columns.  The two groups alternate: while group A turns
-// S_A into P_A on the ALUs, the tensor pipe runs PV_B and the next QK_B, and vice versa.
+// streams the key/value tiles 0..B once for both.  Warp roles (w = warp index):
+//   warps 0-15  softmax warps: tile (w >> 2) & 1, 16 query rows each -- TMEM lanes 32 (w & 3) + 16 (w >> 3)
+//               .. + 15 (a warp may only touch the lane quarter w & 3), read in the 16-lane shapes so that the
+//               four warps of a scheduler work on four disjoint sets of rows
+//   warp  16    TMA producer: Q16/Q8 once, then per key tile the K operand(s) the routing bits ask for
+//               (FP16 and/or INT8) and V, into a ring of equally sized shared-memory chunks
+//   warps 17,18 MMA issuers, one per query tile: tcgen05.mma kind::f16 or kind::i8 for S = Q K^T per the
+//               routing bit, then kind::f16 for O += P V with P read from tensor memory; warp 17 also owns
+//               the TMEM allocation.  The whole warp runs the loop, one elected lane issues.
+//   warp  19    idle
+//   warps 20-23 only in the on-the-fly operand mode: the on-chip quantiser, which makes the INT8 copies of
+//               the query tiles and of the key tiles routed to INT8 in shared memory from the FP16 tiles
+// Tensor memory: S_A | S_B | O_A | O_B (FP32 / INT32 accumulators).  A score tile is produced and consumed in
+// two halves of T/2 key columns; the FP16 probabilities P of a half overwrite the start of that half.  While
+// the softmax warps of a tile turn one half into P, the tensor pipe runs the PV of the other half and the
+// QK^T of the next key tile into it.
 //
 // Every wait is bounded: when one runs out the CTA records a status, raises an abort flag all
 // roles poll, drains what is in flight and returns.
@@ -33,21 +33,27 @@ namespace tilemix {
 
 namespace {
 
-constexpr int kWarpsPerGroup = 4;
-constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
-constexpr int kThreads = 384;             // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
-constexpr int kRegsSoftmax = 216, kRegsOther = 72;   // setmaxnreg split: 2*128*216 + 128*72 = 64512 of the 65536 registers
-// On-the-fly operand mode: a fourth warpgroup, the on-chip quantiser (32 rows of a tile per warp).  512 threads
-// start with 128 registers each; 2*128*200 + 2*128*56 = 65536 stays inside that allotment.
-constexpr int kQuantWarp0 = 12, kQuantWarps = 4;
-constexpr int kThreadsOtf = 512;
-constexpr int kRegsSoftmaxOtf = 200, kRegsOtherOtf = 56;
+constexpr int kSoftmaxWarps = 16;         // 8 per query tile, 16 rows each
+constexpr int kProducerWarp = 16;
+constexpr int kMmaWarp = 17;
+// setmaxnreg only moves registers inside what the block was launched with (threads x registers per thread); an
+// increase beyond that waits for ever.  640 threads start with 96 registers: 512*104 + 128*64 = 61440 = 640*96.
+constexpr int kThreads = 640;
+constexpr int kLaunchRegs = 96;
+constexpr int kRegsSoftmax = 104, kRegsOther = 64;
+// On-the-fly operand mode: a sixth warpgroup, the on-chip quantiser (32 rows of a tile per warp).  768 threads
+// start with 80 registers: 512*96 + 256*48 = 61440 = 768*80.
+constexpr int kQuantWarp0 = 20, kQuantWarps = 4;
+constexpr int kThreadsOtf = 768;
+constexpr int kLaunchRegsOtf = 80;
+constexpr int kRegsSoftmaxOtf = 96, kRegsOtherOtf = 48;
+static_assert(kSoftmaxWarps * 32 * kRegsSoftmax + (kThreads - kSoftmaxWarps * 32) * kRegsOther <= kThreads * kLaunchRegs, "setmaxnreg split");
+static_assert(kSoftmaxWarps * 32 * kRegsSoftmaxOtf + (kThreadsOtf - kSoftmaxWarps * 32) * kRegsOtherOtf <= kThreadsOtf * kLaunchRegsOtf, "setmaxnreg split");
 constexpr uint32_t kQuantBar = 9;         // named barrier of the quantiser warps
 constexpr int kMaxHeadGroup = 8;   // (batch, head) rows whose CTAs are interleaved in the grid order, at most
 constexpr int kRing = 8;
 constexpr int kBundles = 4;        // operand bundles in flight at most (each has a "landed" and a "consumed" barrier)
-constexpr int kWorkspaceClearBytes = 4096;  // status record + optional phase timers
+constexpr int kWorkspaceClearBytes = 4096;  // status record
 constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -128,17 +134,6 @@ struct Ctx {
     int* status;
 };
 
-// Optional phase timers (compile with -DTILEMIX_PHASE_TIMERS): cycles spent in each bounded wait,
-// summed over all CTAs into 64-bit counters that follow the status record in the workspace
-// (index = role * 8 + barrier kind; 32.. = whole-CTA and softmax-loop totals).  Only the first
-// thread of each role contributes.
-#ifdef TILEMIX_PHASE_TIMERS
-#define TM_TIMER_ADD(idx, cycles) atomicAdd(reinterpret_cast<unsigned long long*>(cx.status) + 8 + (idx), \
-                                            static_cast<unsigned long long>(cycles))
-#else
-#define TM_TIMER_ADD(idx, cycles) ((void)0)
-#endif
-
 __device__ __forceinline__ void record_timeout(const Ctx& cx, int role, int tile, int which) {
     *cx.abort_flag = 1;
     if (atomicCAS(&cx.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
@@ -152,9 +147,6 @@ __device__ __forceinline__ void record_timeout(const Ctx& cx, int role, int tile
 __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t parity, int role,
                                          int tile, int which) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
-#ifdef TILEMIX_PHASE_TIMERS
-    const long long c0 = clock64();
-#endif
     const uint64_t t0 = ptx::globaltimer_ns();
     uint32_t it = 0;
     while (!ptx::mbar_try_wait(bar, parity)) {
@@ -166,9 +158,6 @@ __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t p
             }
         }
     }
-#ifdef TILEMIX_PHASE_TIMERS
-    if ((threadIdx.x & 127) == 0 || role >= kRoleProducer) TM_TIMER_ADD((role & 3) * 8 + (which & 7), clock64() - c0);
-#endif
     return true;
 }
 
@@ -208,9 +197,6 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     int skip_word = 0;
     if (threadIdx.x == 0) skip_word = *reinterpret_cast<volatile int*>(prm.status);
 
-#ifdef TILEMIX_PHASE_TIMERS
-    const long long cta_c0 = clock64();
-#endif
     // ---- work item -------------------------------------------------------------------
     // b: batch coordinate of the tensor maps; seq: sequence index (== b for a dense batch);
     // tok0 / len: first token and length of the sequence; row0: its first row among the mask rows
@@ -300,7 +286,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         for (int t = 0; t < 2; ++t) {
             for (int h = 0; h < 2; ++h) {
                 ptx::mbar_init(bar_s(t, h), 1);
-                ptx::mbar_init(bar_p(t, h), kWarpsPerGroup * 32);
+                ptx::mbar_init(bar_p(t, h), kSoftmaxWarps / 2 * 32);
             }
             ptx::mbar_init(bar_pv(t), 1);
             ptx::mbar_init(bar_o(t), 1);
@@ -566,10 +552,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
         // ================================================================ MMA issuers
-        // One issuing thread per query tile (warp kMmaWarp: tile A, the next warp: tile B).  Both walk
-        // the same sequence of ring items; an item goes back to the producer when both have committed it.
+        // One issuing warp per query tile (warp kMmaWarp: tile A, the next warp: tile B); the whole warp runs this
+        // loop with warp-uniform values and stays converged, one elected lane issues each tcgen05 instruction.
+        // Both issuers walk the same sequence of ring items; an item goes back to the producer when both have
+        // committed it.
         ptx::setmaxnreg_dec<OTF ? kRegsOtherOtf : kRegsOther>();
-        if (lane == 0) {
+        {
             const int t = warp - kMmaWarp;
             const int m_t = t ? kB : kA;       // last key tile of this issuer's query tile
             constexpr int TH = C::kTH;
@@ -690,20 +678,21 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             wait_bar(cx, bar_drain, 0, kRoleMma, nkv, kBarDrain);
         }
     } else {
-        // ================================================================ softmax groups
+        // ================================================================ softmax warps
         ptx::setmaxnreg_inc<OTF ? kRegsSoftmaxOtf : kRegsSoftmax>();
-        const int t = warp / kWarpsPerGroup;
+        const int quarter = warp & 3, t = (warp >> 2) & 1, sub = warp >> 3;
         const int m_t = t ? mB : mA;           // query-tile row
         const int k_t = t ? kB : kA;           // its diagonal key tile
         if (t == 0 || hasB) {
-            const int quarter = warp & 3;
-            const int row = quarter * 32 + lane;
-            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            constexpr int TH = C::kTH;         // key columns per half step
+            constexpr int NB = TH / 8;         // blocks of 8 columns per half step
+            // This thread holds two columns (cq, cq + 1 of every block of 8) of the rows rw[0] and rw[1] = rw[0] + 8
+            // of the tile; the four lanes of a quad share a row.
+            const int cq = 2 * (lane & 3);
+            const int rw[2] = {quarter * 32 + sub * 16 + (lane >> 2), quarter * 32 + sub * 16 + (lane >> 2) + 8};
+            const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32 + sub * 16) << 16);
             const uint32_t t_s = lane_base + t * C::kSCols;
             const uint32_t t_o = lane_base + 2 * C::kSCols + t * C::kOCols;
-            const int i_loc = m_t * T + row;                         // row inside the sequence
-            const int64_t i_glob = static_cast<int64_t>(tok0) + i_loc;   // row on the token axis
-            const bool row_valid = row < T && i_loc < len;
             // scales: dense [B,H,T_m] (unit stride over blocks), variable-length [blocks, H]
             const int64_t dk_step = varlen ? prm.Hk : 1;
             float dq = 0.f;
@@ -716,27 +705,19 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                                     : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.ks_blocks;
                 }
             }
-            float m_run = -INFINITY, z = 0.f;
-            float m_seen = -INFINITY;     // largest scaled score seen so far (m_run may lag it)
+            // Shared online-softmax state (Sec. 3.1), log2 domain, per row: running maximum m (identical in the four
+            // lanes of the row's quad), this lane's part of the normaliser z, and the largest score this lane saw.
+            float m_run[2] = {-INFINITY, -INFINITY}, z[2] = {0.f, 0.f}, m_seen[2] = {-INFINITY, -INFINITY};
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
             bool dq_there = !OTF;   // on-the-fly mode: this tile's scale comes from the on-chip quantiser
-
-#ifdef TILEMIX_PHASE_TIMERS
-            const long long loop_c0 = clock64();
-#endif
             float dk_next = (prm.has_int8 && !OTF) ? dk_row[0] : 0.f;
             float a = prm.scale_log2;
             uint32_t int8_route = 0u;
-            constexpr int TH = C::kTH;
             const int n_steps = 2 * (k_t + 1);
-            // One step = one half (TH key columns) of a score tile: while this group works on one half
-            // of S_t, the tensor pipe runs the PV of the previous half and the QK^T of the next one
-            // into the other half.  u = 2*j + h.
-            // While a one-pass step is still computing, the first 32 columns of the next step are put in
-            // flight if that S half is already there (it normally is): `prefetched`.
-            uint32_t first[32];
-            bool prefetched = false;
+            // One step = one half (TH key columns) of a score tile: while the warps of this tile work on one half of
+            // S_t, the tensor pipe runs the PV of the previous half and the QK^T of the next one into the other
+            // half.  u = 2*j + h.
             for (int u = 0; u < n_steps; ++u) {
                 const int j = u >> 1, h = u & 1;
                 if (h == 0) {
@@ -749,15 +730,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     if (!OTF && prm.has_int8 && j < k_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
                 }
                 const uint32_t t_sh = t_s + h * TH;
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long sw0 = clock64();
-#endif
-                if (!prefetched) {
-                    ok = wait_bar(cx, bar_s(t, h), j & 1, role, j, kBarS);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                }
+                ok = wait_bar(cx, bar_s(t, h), j & 1, role, j, kBarS);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                uint32_t s[4 * NB];
+                if constexpr (NB == 8) ptx::tmem_ld16x256_x8(t_sh, s);
+                else ptx::tmem_ld16x256_x4(t_sh, s);
                 if constexpr (OTF) {
                     // the key tile's scale was written by the quantiser before the issuer could start the
                     // MMAs whose result has just been seen
@@ -773,121 +752,113 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         if (a == 0.f) a = 1.f;
                     }
                 }
-#ifdef TILEMIX_PHASE_TIMERS
-                if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(39, clock64() - sw0);
-#endif
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long st0 = clock64();
-#endif
 
-                // ---- shared online-softmax state (Sec. 3.1), log2 domain --------------------------
-                // P = 2^(a*raw - m) is rounded to FP16 and packed two per word into p2[0 .. TH/2).
-                // The running maximum m is lazy: it moves only when a step exceeds it by more than
-                // kTau.  So an interior step is done in ONE pass with the current m, 32 columns at a
-                // time with the next 32 already in flight from tensor memory, while its row maximum is
-                // tracked on the side; only if some row of the warp does exceed m + kTau (rare after
-                // the first tiles) the half tile is re-read and redone in the generic two-pass form.
+                // P = 2^(a*raw - m) is rounded to FP16, one pair per register.  The running maximum m is lazy: an
+                // interior step is done in ONE pass with the current m while the largest score is tracked on the
+                // side; m moves (O and z are rescaled) only after some row of the warp came within kTauHard - kTauSoft
+                // of overflowing FP16, and only if some row of the warp does exceed m + kTauHard the half tile is
+                // redone from the accumulators, which are still in tensor memory, in the generic two-pass form.
                 const bool diag = (j == k_t);
                 bool redo = diag || u == 0 || prm.dbg_n > 0;
-                float alpha = 1.f, sum = 0.f;
+                float alpha[2] = {1.f, 1.f}, sum[2] = {0.f, 0.f};
                 bool grow = false;
-                uint32_t p2[TH / 2];
-                if (__any_sync(0xffffffffu, m_seen > m_run + kTauSoft)) {
+                uint32_t p[2 * NB];
+                if (__any_sync(0xffffffffu, m_seen[0] > m_run[0] + kTauSoft || m_seen[1] > m_run[1] + kTauSoft)) {
                     // Deferred move of the maximum decided on an earlier step (all rows of the warp):
                     // z changes scale here, O~ below together with any move this step itself forces.
-                    const float m_new = fmaxf(m_run, m_seen + kMargin);
-                    alpha = fast_exp2(m_run - m_new);   // 1 for rows that are up to date
-                    m_run = m_new;
-                    z *= alpha;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        m_seen[k] = quad_max(m_seen[k]);
+                        const float m_new = fmaxf(m_run[k], m_seen[k] + kMargin);
+                        alpha[k] = fast_exp2(m_run[k] - m_new);   // 1 for rows that are up to date
+                        m_run[k] = m_new;
+                        z[k] *= alpha[k];
+                    }
                     grow = true;
                 }
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long st1 = clock64();
-#endif
+                ptx::tmem_wait_ld();
                 if (!redo) {
-                    float mx;
-                    if (!prefetched) ptx::tmem_ld32(t_sh, first);
-                    prefetched = false;
-                    // next step: one-pass as well (not the diagonal tile), and its S half ready?
-                    const int jn = (u + 1) >> 1, hn = (u + 1) & 1;
-                    const bool next_fast = u + 1 < n_steps && jn != k_t;
-                    auto late = [&]() {
-                        if (next_fast && __all_sync(0xffffffffu, ptx::mbar_test_wait(bar_s(t, hn), jn & 1))) {
-                            ptx::tc_fence_after_sync();
-                            ptx::tmem_ld32(t_s + hn * TH, first);
-                            prefetched = true;
-                        }
-                    };
-                    if (int8_route) softmax_tile_fast<TH, true>(t_sh, first, a, m_run, p2, sum, mx, late);
-                    else softmax_tile_fast<TH, false>(t_sh, first, a, m_run, p2, sum, mx, late);
-                    const float m_tile = mx * a;
-                    redo = __any_sync(0xffffffffu, m_tile > m_run + kTauHard);   // P would overflow FP16
-                    if (!redo) m_seen = fmaxf(m_seen, m_tile);
+                    float lmax[2];
+                    if (int8_route) softmax_step_fast<NB, true>(s, a, m_run, p, sum, lmax);
+                    else softmax_step_fast<NB, false>(s, a, m_run, p, sum, lmax);
+                    redo = __any_sync(0xffffffffu, lmax[0] > m_run[0] + kTauHard || lmax[1] > m_run[1] + kTauHard);   // P would overflow FP16
+                    if (!redo) {
+                        m_seen[0] = fmaxf(m_seen[0], lmax[0]);
+                        m_seen[1] = fmaxf(m_seen[1], lmax[1]);
+                    }
                 }
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long st2 = clock64() + (__float_as_int(sum) & 0);
-#endif
                 if (redo) {
                     // Generic two-pass form: the very first step, the diagonal tile, steps that move the maximum, and
-                    // every step in debug mode.  The raw accumulators are (still) in tensor memory.
-                    uint32_t s[TH];
-#pragma unroll
-                    for (int c = 0; c < TH / 32; ++c)
-                        ptx::tmem_ld32(t_sh + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-                    ptx::tmem_wait_ld();
+                    // every step in debug mode.
                     if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
                         int idx = -1;
                         if (lane == 0) {
                             for (int e = 0; e < prm.dbg_n; ++e) {
-                                const int32_t* q = prm.dbg_tiles + 4 * e;
-                                if (q[0] == seq && q[1] == hq && q[2] == m_t && q[3] == j) { idx = e; break; }
+                                const int32_t* qd = prm.dbg_tiles + 4 * e;
+                                if (qd[0] == seq && qd[1] == hq && qd[2] == m_t && qd[3] == j) { idx = e; break; }
                             }
                         }
                         idx = __shfl_sync(0xffffffffu, idx, 0);
-                        if (idx >= 0 && row < T) {
-                            int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + row) * T + h * TH;
+                        if (idx >= 0) {
 #pragma unroll
-                            for (int c = 0; c < TH; c += 4)
-                                *reinterpret_cast<uint4*>(dst + c) = make_uint4(s[c], s[c + 1], s[c + 2], s[c + 3]);
-                            if (row == 0) prm.dbg_kind[idx] = static_cast<uint8_t>(int8_route);
+                            for (int k = 0; k < 2; ++k) {
+                                if (rw[k] >= T) continue;
+                                int32_t* dst = prm.dbg_raw + (static_cast<int64_t>(idx) * T + rw[k]) * T + h * TH + cq;
+#pragma unroll
+                                for (int i = 0; i < NB; ++i)
+                                    *reinterpret_cast<uint2*>(dst + 8 * i) = make_uint2(s[4 * i + 2 * k], s[4 * i + 2 * k + 1]);
+                            }
+                            if (rw[0] == 0 && cq == 0) prm.dbg_kind[idx] = static_cast<uint8_t>(int8_route);
                         }
                     }
                     // Common FP32 score domain (App. C), causal legality on the diagonal tile (App. B:
                     // enforced kernel-side, independent of R), row maximum, then the exponentials.
-                    float mx = -INFINITY;
+                    float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c = 0; c < TH; ++c) {
-                        float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
-                        if (diag && h * TH + c > row) v = -INFINITY;
-                        s[c] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
-                    }
-                    const float m_tile = mx * a;     // a >= 0, so max(a*raw) = a*max(raw)
-                    // generic form: move at once (to the largest score seen, this step included)
-                    m_seen = fmaxf(m_seen, m_tile);
-                    float a_now = 1.f;
-                    if (m_seen > m_run + kTauSoft) {
-                        a_now = fast_exp2(m_run - (m_seen + kMargin));
-                        m_run = m_seen + kMargin;
-                        grow = true;
-                    }
-                    const float2 a2 = make_float2(a, a), nm2 = make_float2(-m_run, -m_run);
-                    float2 acc = make_float2(0.f, 0.f);
+                    for (int i = 0; i < NB; ++i) {
 #pragma unroll
-                    for (int c = 0; c < TH; c += 2) {
-                        const float2 t2 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), a2, nm2);
-                        const float2 pp = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
-                        acc = __fadd2_rn(acc, pp);
-                        p2[c >> 1] = pack_half2(pp.x, pp.y);
+                        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const int c = 4 * i + 2 * k + e;
+                                float v = int8_route ? __int2float_rn(static_cast<int>(s[c])) : __uint_as_float(s[c]);
+                                if (diag && h * TH + 8 * i + cq + e > rw[k]) v = -INFINITY;
+                                s[c] = __float_as_uint(v);
+                                mx[k] = fmaxf(mx[k], v);
+                            }
+                        }
                     }
-                    sum = acc.x + acc.y;
-                    z *= a_now;
-                    alpha *= a_now;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        // generic form: move at once (to the largest score seen, this step included)
+                        m_seen[k] = quad_max(fmaxf(m_seen[k], mx[k] * a));     // a >= 0, so max(a*raw) = a*max(raw)
+                        float a_now = 1.f;
+                        if (m_seen[k] > m_run[k] + kTauSoft) {
+                            a_now = fast_exp2(m_run[k] - (m_seen[k] + kMargin));
+                            m_run[k] = m_seen[k] + kMargin;
+                            grow = true;
+                        }
+                        z[k] *= a_now;
+                        alpha[k] *= a_now;
+                    }
+                    const float2 a2 = make_float2(a, a);
+                    float2 acc[2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+                    for (int i = 0; i < NB; ++i) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+                            const float2 t2 = __ffma2_rn(make_float2(__uint_as_float(s[4 * i + 2 * k]), __uint_as_float(s[4 * i + 2 * k + 1])),
+                                                         a2, make_float2(-m_run[k], -m_run[k]));
+                            const float2 pp = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
+                            acc[k] = __fadd2_rn(acc[k], pp);
+                            p[2 * i + k] = pack_half2(pp.x, pp.y);
+                        }
+                    }
+                    sum[0] = acc[0].x + acc[0].y;
+                    sum[1] = acc[1].x + acc[1].y;
                 }
-                z += sum;
-#ifdef TILEMIX_PHASE_TIMERS
-                const long long st3 = clock64() + (__float_as_int(z) & 0);
-#endif
+                z[0] += sum[0];
+                z[1] += sum[1];
 
                 if (u > 0 && __any_sync(0xffffffffu, grow)) {
                     // O~ *= alpha.  The PV of the previous step may still be accumulating into O~: wait
@@ -900,76 +871,61 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     ptx::tc_fence_after_sync();
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
-                        uint32_t o[32];
-                        ptx::tmem_ld32(t_o + c * 32, o);
+                        uint32_t o[16];
+                        ptx::tmem_ld16x256_x4(t_o + c * 32, o);
                         ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        ptx::tmem_st32(t_o + c * 32, o);
+                        for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha[(e >> 1) & 1]);
+                        ptx::tmem_st16x256_x4(t_o + c * 32, o);
                     }
                 }
-                if constexpr (TH / 2 == 32) {
-                    ptx::tmem_st32(t_sh, p2);
-                } else {
-                    ptx::tmem_st16(t_sh, p2);
-                }
+                if constexpr (NB == 8) ptx::tmem_st16x128_x8(t_sh, p);
+                else ptx::tmem_st16x128_x4(t_sh, p);
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t, h));
-#ifdef TILEMIX_PHASE_TIMERS
-                if ((threadIdx.x & 127) == 0) {
-                    const long long st4 = clock64();
-
-                    TM_TIMER_ADD(40, st1 - st0); TM_TIMER_ADD(41, st2 - st1); TM_TIMER_ADD(42, st3 - st2);
-                    TM_TIMER_ADD(43, st4 - st3); TM_TIMER_ADD(44, 1);
-                }
-#endif
             }
 
-#ifdef TILEMIX_PHASE_TIMERS
-            if ((threadIdx.x & 127) == 0) TM_TIMER_ADD(33 + t, clock64() - loop_c0);
-#endif
             if (ok) {
                 ok = wait_bar(cx, bar_o(t), 0, role, k_t + 1, kBarO);
                 ok = __all_sync(0xffffffffu, ok);
             }
             if (ok) {
+                // Finalise (Sec. 3.1): O = O~ / z in FP16; LSE = m + ln z.
                 ptx::tc_fence_after_sync();
-                const float inv = 1.f / z;
-                __half* dst = prm.out + b * prm.os[0] + hq * prm.os[1] + i_glob * prm.os[2];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const float z_row = quad_sum(z[k]);
+                    const int i_loc = m_t * T + rw[k];                            // row inside the sequence
+                    const int64_t i_glob = static_cast<int64_t>(tok0) + i_loc;    // row on the token axis
+                    const bool row_valid = rw[k] < T && i_loc < len;
+                    z[k] = row_valid ? 1.f / z_row : 0.f;
+                    if (row_valid && cq == 0 && prm.lse != nullptr)
+                        prm.lse[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.L + i_glob] = (m_run[k] + log2f(z_row)) * kLn2;
+                }
+                __half* dst0 = prm.out + b * prm.os[0] + hq * prm.os[1] + (static_cast<int64_t>(tok0) + m_t * T) * prm.os[2] + cq;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    ptx::tmem_ld32(t_o + c * 32, o);
+                    uint32_t o[16];
+                    ptx::tmem_ld16x256_x4(t_o + c * 32, o);
                     ptx::tmem_wait_ld();
-                    if (row_valid) {
 #pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            uint32_t h[4];
+                    for (int k = 0; k < 2; ++k) {
+                        if (z[k] == 0.f) continue;     // a row beyond the sequence (or the 64-row tile): not written
+                        __half* dst = dst0 + rw[k] * prm.os[2] + c * 32;
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const __half2 hv = __floats2half2_rn(__uint_as_float(o[e + 2 * u]) * inv,
-                                                                     __uint_as_float(o[e + 2 * u + 1]) * inv);
-                                h[u] = *reinterpret_cast<const uint32_t*>(&hv);
-                            }
-                            *reinterpret_cast<uint4*>(dst + c * 32 + e) = make_uint4(h[0], h[1], h[2], h[3]);
+                        for (int i = 0; i < 4; ++i) {
+                            const __half2 hv = __floats2half2_rn(__uint_as_float(o[4 * i + 2 * k]) * z[k],
+                                                                 __uint_as_float(o[4 * i + 2 * k + 1]) * z[k]);
+                            *reinterpret_cast<__half2*>(dst + 8 * i) = hv;
                         }
                     }
                 }
-                if (row_valid && prm.lse != nullptr)
-                    prm.lse[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.L + i_glob] = (m_run + log2f(z)) * kLn2;
             }
         }
     }
 
     // ---- teardown -----------------------------------------------------------------------
-#ifdef TILEMIX_PHASE_TIMERS
-    if (threadIdx.x == 0) {
-        TM_TIMER_ADD(32, clock64() - cta_c0);
-        TM_TIMER_ADD(35, 1);
-        TM_TIMER_ADD(36, nkv);
-    }
-#endif
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) {
@@ -1076,6 +1032,12 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
                             : static_cast<int64_t>(g.B) * g.Hq * ((g.T_m + 1) / 2);
     if (ctas == 0) return TILEMIX_OK;   // only zero-length sequences
     if (ctas > 0x7fffffffLL) return static_cast<int>(cudaErrorInvalidConfiguration);
+    // The register split inside the kernel (setmaxnreg) assumes what the block is launched with; a build that
+    // gave the kernel fewer registers must not run (an increase beyond the block's allotment never returns).
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, kernel);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    if (fa.numRegs < (otf ? kLaunchRegsOtf : kLaunchRegs)) return TILEMIX_ERR_UNSUPPORTED;
     kernel<<<static_cast<unsigned>(ctas), otf ? kThreadsOtf : kThreads, C::kSmemAlloc, stream>>>(prm, tq, tk, tv, tq8, tk8);
     g_launch_count.fetch_add(1);
     return static_cast<int>(cudaGetLastError());
