@@ -58,15 +58,18 @@ constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory
 constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-// Lazy rescale.  P = 2^(score - m) is handed to the tensor pipe in FP16, so the running maximum m
-// may lag the true row maximum by up to kTauHard powers of two (P <= 2^15 fits; z and O are FP32).
-// A tile whose rows stay within kTauHard of m is never recomputed.  m is kept kMargin ABOVE the largest
-// score seen (P then tops out at 2^-kMargin, still 18 binades above the smallest FP16 subnormal), so a
-// later score has to beat everything before it by 2^(kTauHard + kMargin) to force a recomputation.
-// When some row of a warp got more than kTauSoft above its m, every row of that warp moves its m
-// *after* the tile (O and z are rescaled before the next one): that restores the headroom without
-// touching probabilities already computed, and one pass over O serves all 32 rows.
-constexpr float kTauSoft = 8.0f, kTauHard = 15.0f, kMargin = 6.0f;
+// Lazy running maximum.  P = 2^(score - m) is handed to the tensor pipe in FP16 (largest finite value just
+// below 2^16), z and O are FP32, so m may lag the true row maximum.  An interior step is done in one pass with
+// the current m and is accepted when this thread's part of each row sum stays below 2^kAccept (no probability
+// of the step can then exceed 2^kAccept).  Otherwise the step is redone from the accumulators in the generic
+// two-pass form, which moves m to kMargin above the step's maximum whenever that maximum is more than kMove above
+// m (a rejected step always is: 2^kAccept spread over at most 16 values) and rescales z and O.  After a move
+// P tops out at 2^-kMargin, 18 binades above the smallest FP16 subnormal, and a later score has to beat
+// everything before it by 2^(kMove + kMargin) to move m again.
+constexpr float kAccept = 8.0f, kMove = 4.0f, kMargin = 6.0f;
+// the INT8 route leaves the conversion bias to the scaling FMA while a * 1.5*2^23 <= kFoldLimit: the addend
+// m + a*1.5*2^23 is then below 2^13 and its rounding moves a score by at most 2^-12 (a relative 1.7e-4 in P)
+constexpr float kFoldLimit = 4096.0f;
 
 enum Role : int { kRoleSoftmaxA = 0, kRoleSoftmaxB = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQuant = 4 };
 enum Bar : int { kBarQ = 0, kBarRingFull = 1, kBarRingEmpty = 2, kBarS = 3, kBarP = 4, kBarO = 5, kBarDrain = 6, kBarPV = 7,
@@ -706,8 +709,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 }
             }
             // Shared online-softmax state (Sec. 3.1), log2 domain, per row: running maximum m (identical in the four
-            // lanes of the row's quad), this lane's part of the normaliser z, and the largest score this lane saw.
-            float m_run[2] = {-INFINITY, -INFINITY}, z[2] = {0.f, 0.f}, m_seen[2] = {-INFINITY, -INFINITY};
+            // lanes of the row's quad) and this lane's part of the normaliser z.
+            float m_run[2] = {-INFINITY, -INFINITY}, z[2] = {0.f, 0.f};
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
             bool dq_there = !OTF;   // on-the-fly mode: this tile's scale comes from the on-chip quantiser
@@ -753,39 +756,26 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     }
                 }
 
-                // P = 2^(a*raw - m) is rounded to FP16, one pair per register.  The running maximum m is lazy: an
-                // interior step is done in ONE pass with the current m while the largest score is tracked on the
-                // side; m moves (O and z are rescaled) only after some row of the warp came within kTauHard - kTauSoft
-                // of overflowing FP16, and only if some row of the warp does exceed m + kTauHard the half tile is
-                // redone from the accumulators, which are still in tensor memory, in the generic two-pass form.
+                // P = 2^(a*raw - m) is rounded to FP16, one pair per register.
                 const bool diag = (j == k_t);
                 bool redo = diag || u == 0 || prm.dbg_n > 0;
                 float alpha[2] = {1.f, 1.f}, sum[2] = {0.f, 0.f};
                 bool grow = false;
                 uint32_t p[2 * NB];
-                if (__any_sync(0xffffffffu, m_seen[0] > m_run[0] + kTauSoft || m_seen[1] > m_run[1] + kTauSoft)) {
-                    // Deferred move of the maximum decided on an earlier step (all rows of the warp):
-                    // z changes scale here, O~ below together with any move this step itself forces.
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        m_seen[k] = quad_max(m_seen[k]);
-                        const float m_new = fmaxf(m_run[k], m_seen[k] + kMargin);
-                        alpha[k] = fast_exp2(m_run[k] - m_new);   // 1 for rows that are up to date
-                        m_run[k] = m_new;
-                        z[k] *= alpha[k];
-                    }
-                    grow = true;
-                }
                 ptx::tmem_wait_ld();
                 if (!redo) {
-                    float lmax[2];
-                    if (int8_route) softmax_step_fast<NB, true>(s, a, m_run, p, sum, lmax);
-                    else softmax_step_fast<NB, false>(s, a, m_run, p, sum, lmax);
-                    redo = __any_sync(0xffffffffu, lmax[0] > m_run[0] + kTauHard || lmax[1] > m_run[1] + kTauHard);   // P would overflow FP16
-                    if (!redo) {
-                        m_seen[0] = fmaxf(m_seen[0], lmax[0]);
-                        m_seen[1] = fmaxf(m_seen[1], lmax[1]);
+                    if (!int8_route) {
+                        const float addend[2] = {-m_run[0], -m_run[1]};
+                        softmax_step_fast<NB, kFp32>(s, a, addend, p, sum);
+                    } else if (a * kInt8Bias <= kFoldLimit) {
+                        // one explicit FMA: every instantiation of the kernel rounds the addend the same way
+                        const float addend[2] = {-__fmaf_rn(a, kInt8Bias, m_run[0]), -__fmaf_rn(a, kInt8Bias, m_run[1])};
+                        softmax_step_fast<NB, kInt8Folded>(s, a, addend, p, sum);
+                    } else {
+                        const float addend[2] = {-m_run[0], -m_run[1]};
+                        softmax_step_fast<NB, kInt8Exact>(s, a, addend, p, sum);
                     }
+                    redo = __any_sync(0xffffffffu, !(sum[0] <= exp2f(kAccept) && sum[1] <= exp2f(kAccept)));   // also true for a NaN
                 }
                 if (redo) {
                     // Generic two-pass form: the very first step, the diagonal tile, steps that move the maximum, and
@@ -830,16 +820,13 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     }
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
-                        // generic form: move at once (to the largest score seen, this step included)
-                        m_seen[k] = quad_max(fmaxf(m_seen[k], mx[k] * a));     // a >= 0, so max(a*raw) = a*max(raw)
-                        float a_now = 1.f;
-                        if (m_seen[k] > m_run[k] + kTauSoft) {
-                            a_now = fast_exp2(m_run[k] - (m_seen[k] + kMargin));
-                            m_run[k] = m_seen[k] + kMargin;
+                        const float m_step = quad_max(mx[k] * a);     // a >= 0, so max(a*raw) = a*max(raw)
+                        if (m_step > m_run[k] + kMove) {
+                            alpha[k] = fast_exp2(m_run[k] - (m_step + kMargin));
+                            m_run[k] = m_step + kMargin;
+                            z[k] *= alpha[k];
                             grow = true;
                         }
-                        z[k] *= a_now;
-                        alpha[k] *= a_now;
                     }
                     const float2 a2 = make_float2(a, a);
                     float2 acc[2] = {{0.f, 0.f}, {0.f, 0.f}};

@@ -42,43 +42,44 @@ __device__ __forceinline__ float quad_sum(float v) {
     return v + __shfl_xor_sync(0xffffffffu, v, 2);
 }
 
+// How the raw accumulators of a step become floats: FP32 scores as they are; INT32 scores by the bias trick --
+// bits(1.5*2^23) + i is the float 1.5*2^23 + i for |i| < 2^22 (here |i| <= 127*127*D) -- either with the bias
+// removed by an exact subtraction before the scaling (kInt8Exact), or left in and cancelled by the addend of the
+// scaling FMA, a*(1.5*2^23 + i) - (m + a*1.5*2^23) (kInt8Folded: one instruction less per pair; the addend is
+// rounded once per step, so the caller uses it only while that rounding is negligible).
+enum ScoreKind : int { kFp32 = 0, kInt8Exact = 1, kInt8Folded = 2 };
+constexpr float kInt8Bias = 12582912.f;   // 1.5 * 2^23
+
 // One interior step (NB blocks of 8 key columns, no causal mask) in one pass with the current running
 // maxima: raw accumulators s -> P = 2^(a*raw - m) rounded to FP16 (p[2i + k] = the pair of row k in block
-// i), this thread's part of the FP32 row sums and of the row maxima of a*raw.  INT32 accumulators are made
-// floats without the conversion unit: bits(1.5*2^23) + i is the float 1.5*2^23 + i for |i| < 2^22 (here
-// |i| <= 127*127*D), and subtracting 1.5*2^23 is exact.
-template <int NB, bool INT8>
-__device__ __forceinline__ void softmax_step_fast(const uint32_t (&s)[4 * NB], float a, const float (&m_run)[2],
-                                                  uint32_t (&p)[2 * NB], float (&sum)[2], float (&lmax)[2]) {
+// i) and this thread's part of the FP32 row sums.  addend[k] = -m_k (kFp32, kInt8Exact) or -(m_k + a*1.5*2^23)
+// (kInt8Folded).
+template <int NB, int KIND>
+__device__ __forceinline__ void softmax_step_fast(const uint32_t (&s)[4 * NB], float a, const float (&addend)[2],
+                                                  uint32_t (&p)[2 * NB], float (&sum)[2]) {
     const float2 a2 = make_float2(a, a);
-    const float2 unbias = make_float2(-12582912.f, -12582912.f);
+    const float2 unbias = make_float2(-kInt8Bias, -kInt8Bias);
     float2 acc[2] = {{0.f, 0.f}, {0.f, 0.f}};
-    int mi[2] = {INT_MIN, INT_MIN};
-    float mf[2] = {-INFINITY, -INFINITY};
 #pragma unroll
     for (int i = 0; i < NB; ++i) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const uint32_t r0 = s[4 * i + 2 * k], r1 = s[4 * i + 2 * k + 1];
             float2 x;
-            if (INT8) {
-                mi[k] = __vimax3_s32(mi[k], static_cast<int>(r0), static_cast<int>(r1));
-                x = __fadd2_rn(make_float2(__uint_as_float(r0 + 0x4B400000u), __uint_as_float(r1 + 0x4B400000u)), unbias);
-            } else {
+            if (KIND == kFp32) {
                 x = make_float2(__uint_as_float(r0), __uint_as_float(r1));
-                mf[k] = fmax3(mf[k], x.x, x.y);
+            } else {
+                x = make_float2(__uint_as_float(r0 + 0x4B400000u), __uint_as_float(r1 + 0x4B400000u));
+                if (KIND == kInt8Exact) x = __fadd2_rn(x, unbias);
             }
-            const float2 t2 = __ffma2_rn(x, a2, make_float2(-m_run[k], -m_run[k]));
+            const float2 t2 = __ffma2_rn(x, a2, make_float2(addend[k], addend[k]));
             const float2 e = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
             acc[k] = __fadd2_rn(acc[k], e);
             p[2 * i + k] = pack_half2(e.x, e.y);
         }
     }
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        sum[k] = acc[k].x + acc[k].y;
-        lmax[k] = a * (INT8 ? __int2float_rn(mi[k]) : mf[k]);   // a >= 0: max(a*raw) = a*max(raw)
-    }
+    sum[0] = acc[0].x + acc[0].y;
+    sum[1] = acc[1].x + acc[1].y;
 }
 
 }  // namespace tilemix
