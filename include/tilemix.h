@@ -177,7 +177,11 @@ int tilemix_attention_fwd_noalloc(const tilemix_problem_t* p, const void* q_f16,
  * `stream` is made to wait for the last copy, so synchronising `stream` completes the call.
  *   q_host,k_host,v_host  host FP16, dense [B,H,L,d];  route_host host uint8 [nb,Hk,T_m,T_mask]
  *   out_host              host FP16, dense [B,Hq,L,d]
- *   arena                 device scratch of >= tilemix_arena_size(p) bytes, 256-byte aligned */
+ *   arena                 device scratch of >= tilemix_arena_size(p) bytes, 256-byte aligned
+ * Host threads: the helper streams and events are one set per device, and a call holds a per-device lock of
+ * the library while it enqueues, so calls from several host threads on one device (each with its own arena,
+ * output buffer and stream) are safe and are enqueued one whole call after the other; their copies share the
+ * two helper streams and therefore run in that order.  The call does not synchronise anything. */
 int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const void* k_host,
                          const void* v_host, const uint8_t* route_host, uint32_t pack_flags,
                          void* out_host, void* arena, size_t arena_bytes, void* stream);
@@ -216,7 +220,11 @@ typedef struct tilemix_varlen {
 /* Derived sizes of a variable-length batch, out = {total tokens, sum T_m, sum blocks of Q,
  * sum blocks of K, T_mask_max, W, longest sequence}.  Returns TILEMIX_OK or a negative error. */
 int tilemix_varlen_counts(const tilemix_problem_t* p, const tilemix_varlen_t* vl, int64_t out[7]);
-/* Bytes of `workspace` the three calls below need (0 on invalid arguments): the 4096-byte
+/* The three calls below copy their prefix-sum tables from a host buffer of the call (pageable memory) to the
+ * workspace with cudaMemcpyAsync: do not call them while `stream` is being captured into a CUDA graph (the graph
+ * would keep a pointer to memory that is gone when the call returns), and expect the copy to be staged by the
+ * driver like any copy from pageable memory.
+ * Bytes of `workspace` the three calls below need (0 on invalid arguments): the 4096-byte
  * status area of tilemix_attention_fwd followed by the prefix-sum tables and the attention
  * kernel's work list (two int32 per pair of query tiles).  Every call copies
  * the tables into its workspace on `stream`, so one workspace may serve all three calls in
@@ -273,8 +281,10 @@ typedef struct tilemix_decode {
  * and the partial results of the splits (0 on an invalid problem). */
 size_t tilemix_decode_workspace_size(const tilemix_decode_t* p);
 /*   q_f16      FP16 [B, Hq, d]
- *   k_f16      FP16 [B, Hk, max_len, d]   (may be NULL if every legal group is INT8-routed:
- *                                          a 0 bit then reads NULL -- the caller's contract)
+ *   k_f16      FP16 [B, Hk, max_len, d]   (may be NULL if every group inside the cache lengths is
+ *                                          INT8-routed; a 0 bit there is then found by the kernel before it
+ *                                          reads anything: no access is made, the status record of the
+ *                                          workspace reads TILEMIX_ERR_NULL and the outputs are undefined)
  *   k_i8, v_i8 INT8 [B, Hk, max_len, d];  k_scale, v_scale FP32 [B, Hk, ceil(max_len/tile_n)]
  *   mask_words uint32 [nb, Hk, W], W = ceil(ceil(max_len/(G*tile_n))/32); NULL = all FP16
  *   cache_len  int32 [B] on the DEVICE, 0 <= cache_len[b] <= max_len (values outside are clamped to that
@@ -283,7 +293,9 @@ size_t tilemix_decode_workspace_size(const tilemix_decode_t* p);
  *   out_f16    FP16 [B, Hq, d];  lse nullable FP32 [B, Hq]
  *   q_i8_out / q_scale_out  nullable INT8 [B, Hq, d] / FP32 [B, Hq]: the quantised query the
  *              kernel used (for checking)
- * Two kernels are enqueued on `stream`.  Errors as for the other entry points. */
+ * Three kernels are enqueued on `stream` (preparation of the lengths and the status record, the step over the
+ * splits, the merge).  Errors as for the other entry points; tilemix_read_status on the workspace reports what the
+ * kernel itself found (a bounded wait that ran out, or the missing FP16 cache above). */
 int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const void* k_f16,
                           const int8_t* k_i8, const float* k_scale, const int8_t* v_i8,
                           const float* v_scale, const uint32_t* mask_words,

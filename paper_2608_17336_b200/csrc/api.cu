@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace tilemix {
@@ -44,6 +46,36 @@ int check_device() {
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// What tilemix_attention_fwd and tilemix_attention_fwd_chunk check on the host before the launch (the geometry is
+// resolved by the caller: the chunk entry point rewrites the key/value side of it first).
+int checked_attention(const Geometry& g, const void* q_f16, const void* k_f16, const void* v_f16, const int8_t* q_i8,
+                      const int8_t* k_i8, const float* q_scale, const float* k_scale, const uint32_t* mask_words,
+                      void* out_f16, float* lse, void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg,
+                      void* stream) {
+    if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
+    const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
+    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;   // INT8 operands and scales are made on chip
+    if (!force16 && !otf && !(q_i8 && k_i8 && q_scale && k_scale)) return TILEMIX_ERR_NULL;
+    if (!force16 && !mask_words) return TILEMIX_ERR_NULL;
+    if (otf && !(g.d == 128 && g.tile_m == 128 && g.tile_n == 128)) return TILEMIX_ERR_UNSUPPORTED;
+    if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
+    if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
+    const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
+                          (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
+    if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
+    if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
+        !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
+        (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
+        return TILEMIX_ERR_ALIGN;
+    if (workspace_bytes < kStatusAreaBytes) return TILEMIX_ERR_WORKSPACE;
+    const int rc = check_device();
+    if (rc) return rc;
+    return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
+                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+}
 
 }  // namespace
 
@@ -116,27 +148,8 @@ int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const v
     Geometry g;
     int rc = resolve(p, &g);
     if (rc) return rc;
-    if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
-    const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
-    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;   // INT8 operands and scales are made on chip
-    if (!force16 && !otf && !(q_i8 && k_i8 && q_scale && k_scale)) return TILEMIX_ERR_NULL;
-    if (!force16 && !mask_words) return TILEMIX_ERR_NULL;
-    if (otf && !(g.d == 128 && g.tile_m == 128 && g.tile_n == 128)) return TILEMIX_ERR_UNSUPPORTED;
-    if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
-    if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
-    const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
-                          (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
-    if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
-    if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
-        !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
-        (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
-        return TILEMIX_ERR_ALIGN;
-    if (workspace_bytes < tilemix_workspace_size(p)) return TILEMIX_ERR_WORKSPACE;
-    if ((rc = check_device())) return rc;
-    return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
-                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+    return checked_attention(g, q_f16, k_f16, v_f16, q_i8, k_i8, q_scale, k_scale, mask_words, out_f16, lse, workspace,
+                             workspace_bytes, dbg, stream);
 }
 
 int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, const void* q_f16, const void* k_f16,
@@ -160,27 +173,8 @@ int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, cons
     g.ks_blocks = static_cast<int>(ceil_div(kv_len, g.blk_k));
     g.T_mask = static_cast<int>(ceil_div(kv_len, static_cast<int64_t>(g.G) * g.tile_n));
     g.W = static_cast<int>(ceil_div(g.T_mask, 32));
-    if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
-    const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
-    const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;
-    if (!force16 && !otf && !(q_i8 && k_i8 && q_scale && k_scale)) return TILEMIX_ERR_NULL;
-    if (!force16 && !mask_words) return TILEMIX_ERR_NULL;
-    if (otf && !(g.d == 128 && g.tile_m == 128 && g.tile_n == 128)) return TILEMIX_ERR_UNSUPPORTED;
-    if (dbg && dbg->n_tiles > 0 && !(dbg->tiles && dbg->raw && dbg->kind)) return TILEMIX_ERR_NULL;
-    if (dbg && dbg->n_tiles < 0) return TILEMIX_ERR_SHAPE;
-    const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
-                          (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
-    if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
-    if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
-        !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
-        (dbg && dbg->n_tiles > 0 && !aligned16(dbg->raw)))
-        return TILEMIX_ERR_ALIGN;
-    if (workspace_bytes < 4096) return TILEMIX_ERR_WORKSPACE;
-    if ((rc = check_device())) return rc;
-    return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
-                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+    return checked_attention(g, q_f16, k_f16, v_f16, q_i8, k_i8, q_scale, k_scale, mask_words, out_f16, lse, workspace,
+                             workspace_bytes, dbg, stream);
 }
 
 int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {
@@ -192,7 +186,7 @@ int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {
 size_t tilemix_workspace_size(const tilemix_problem_t* p) {
     Geometry g;
     if (resolve(p, &g)) return 0;
-    return 4096;   // status record (16 bytes) + optional phase timers / trace
+    return kStatusAreaBytes;   // status record (16 bytes) at the start
 }
 
 size_t tilemix_scratch_bytes(const tilemix_problem_t* p) {
@@ -244,15 +238,11 @@ struct HostPipe {
     cudaEvent_t start = nullptr, landed[kMaxChunks] = {}, done[kMaxChunks] = {}, drained = nullptr;
 };
 HostPipe g_pipe[64];
-std::atomic<int> g_pipe_lock{0};
+std::mutex g_pipe_mutex[64];   // one call at a time per device enqueues on the helper streams
 
-int host_pipe(HostPipe** out) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return static_cast<int>(e);
-    if (dev < 0 || dev >= 64) return TILEMIX_ERR_UNSUPPORTED;
+// Called with g_pipe_mutex[dev] held.
+int host_pipe(int dev, HostPipe** out) {
     HostPipe& hp = g_pipe[dev];
-    while (g_pipe_lock.exchange(1, std::memory_order_acquire) != 0) {}
     int rc = TILEMIX_OK;
     if (!hp.ready) {
         auto ev = [&](cudaEvent_t* x) { if (rc == 0) rc = static_cast<int>(cudaEventCreateWithFlags(x, cudaEventDisableTiming)); };
@@ -262,7 +252,6 @@ int host_pipe(HostPipe** out) {
         for (int i = 0; i < kMaxChunks; ++i) { ev(&hp.landed[i]); ev(&hp.done[i]); }
         hp.ready = rc == 0;
     }
-    g_pipe_lock.store(0, std::memory_order_release);
     *out = &hp;
     return rc;
 }
@@ -283,8 +272,14 @@ int tilemix_prefill_host(const tilemix_problem_t* p, const void* q_host, const v
     if (arena_bytes < a.total) return TILEMIX_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* base = static_cast<uint8_t*>(arena);
+    // The helper streams and events belong to the device, so the whole enqueue below is one critical section per
+    // device: calls from several host threads (on any streams) are enqueued one after the other, never interleaved.
+    int dev = 0;
+    if (cudaError_t de = cudaGetDevice(&dev); de != cudaSuccess) return static_cast<int>(de);
+    if (dev < 0 || dev >= 64) return TILEMIX_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> enqueue_lock(g_pipe_mutex[dev]);
     HostPipe* hp = nullptr;
-    if ((rc = host_pipe(&hp))) return rc;
+    if ((rc = host_pipe(dev, &hp))) return rc;
 
     // The batch (or, for one sequence, its KV heads) is cut into chunks that flow through three
     // engines at once: host->device copies on a helper stream, the three kernels on the caller's

@@ -1087,9 +1087,10 @@ extern "C" int tilemix_attention_fwd_noalloc(const tilemix_problem_t* p, const v
                                              const tilemix_debug_t* dbg, void** workspace_out, void* stream) {
     using namespace tilemix;
     if (p == nullptr || !q_f16 || !k_f16 || !v_f16 || !out_f16) return TILEMIX_ERR_NULL;
-    const size_t need = tilemix_workspace_size(p);
-    if (need == 0) return TILEMIX_ERR_SHAPE;
-    if (need > kStaticWorkspaceBytes) return TILEMIX_ERR_WORKSPACE;   // beyond the fixed scratch
+    Geometry g;
+    const int bad = resolve(p, &g);      // the codes tilemix_attention_fwd returns for the same problem
+    if (bad) return bad;
+    if (tilemix_workspace_size(p) > kStaticWorkspaceBytes) return TILEMIX_ERR_WORKSPACE;   // beyond the fixed scratch
     void* ws = nullptr;
     const int rc = static_workspace(&ws);
     if (rc != TILEMIX_OK) return rc;

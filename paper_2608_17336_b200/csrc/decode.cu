@@ -192,7 +192,21 @@ decode_kernel(const DecodeParams prm) {
         // delta_K >= 0; the FP16 route is marked by a negative x (its delta_K is not used)
         meta[i] = make_float2(route_of(tile) ? dk[tile / per_blk] : -1.f, dv[tile / per_blk]);
     }
-    __syncthreads();   // barriers initialised, query rows and tile metadata staged
+    if constexpr (!F16K) {
+        // This instance was chosen because no FP16 key cache was passed: every group inside the cache length has
+        // to be INT8-routed.  A 0 bit is found here, before any copy is started; the CTA records it and leaves
+        // (no access is made, nothing is in flight).
+        int fp16_group = 0;
+        for (int tile = t0 + tid; tile < t1; tile += kDecodeThreads) fp16_group |= route_of(tile) ? 0 : 1;
+        if (__syncthreads_or(fp16_group)) {
+            if (tid == 0 && atomicCAS(&prm.status[0], 0, TILEMIX_ERR_NULL) == 0) {
+                prm.status[1] = 16; prm.status[2] = t0; prm.status[3] = 1;
+            }
+            return;
+        }
+    } else {
+        __syncthreads();   // barriers initialised, query rows and tile metadata staged
+    }
 
     // per-warp flash-decoding state: rows g (< R) of this warp's keys
     float m_run = -INFINITY, z_part = 0.f;          // z_part: this lane's share of the row sum

@@ -46,6 +46,9 @@ def _check(q, k, v, route, lens, tile, G, **kw):
     # the cache itself: the library quantiser against the oracle's (bit-exact)
     k8_ref, ks_ref = oracle.quantize(k16, tile)
     assert np.array_equal(cache["k8"], k8_ref) and np.array_equal(cache["ks"].view(np.uint32), ks_ref.view(np.uint32))
+    v16 = np.ascontiguousarray(v.view(torch.int16).numpy()).view(np.uint16)
+    v8_ref, vs_ref = oracle.quantize(v16, tile)      # the V cache too, before the oracle is given it
+    assert np.array_equal(cache["v8"], v8_ref) and np.array_equal(cache["vs"].view(np.uint32), vs_ref.view(np.uint32))
     q8_ref, dq_ref = od.quantize_query(q16)
     assert np.array_equal(res["q8"].cpu().numpy(), q8_ref)
     assert np.array_equal(res["q_scale"].cpu().numpy().view(np.uint32), dq_ref.view(np.uint32))
@@ -137,3 +140,32 @@ def test_decode_out_of_range_lengths_are_clamped():
     bad, _ = _gpu(q, k, v, route, np.asarray([100000, -5, 123], np.int32), 128, 1)
     assert torch.equal(good["out"].view(torch.int16), bad["out"].view(torch.int16))
     assert torch.equal(good["lse"], bad["lse"])
+
+
+def test_decode_without_fp16_cache_reports_an_fp16_routed_group():
+    """No FP16 key cache is passed but one group inside the cache length is routed to FP16: the kernel must find
+    that before it reads anything and say so in the status record (no fault); the same workspace then serves a
+    correct call."""
+    from paper_2608_17336_b200 import binding as tm
+    dev = torch.device("cuda:0")
+    q, k, v, route, lens = _case(2, 4, 2, 700, 128, 128, 1, seed=51, lens=[700, 300], f8=1.0)
+    route[:] = 1
+    B, Hq, d = q.shape
+    Hk, L = k.shape[1], k.shape[2]
+    kd, vd = k.to(dev), v.to(dev)
+    k8, v8, ks, vs = tm.tilemix_quantize_qk(tm.problem(B, Hk, Hk, L, d, 128, 128), kd, vd)
+    p = tm.decode_problem(B, Hq, Hk, d, L, 128, 1)
+    bad = route.copy()
+    bad[0, 1, 3] = 0                                     # keys 384..511 of KV head 1: inside both cache lengths? (300 < 384: batch 0 only)
+    for r, want in ((bad, tm.ERR_NULL), (route, 0)):
+        words = torch.from_numpy(od.pack_row(r).view(np.int32)).to(dev)
+        res = tm.tilemix_decode_int8kv(p, q.to(dev), None, k8, ks, v8, vs, words, torch.from_numpy(lens).to(dev))
+        code, rec = tm.tilemix_read_status(res["workspace"])
+        assert code == want, rec
+    # a 0 bit beyond every cache length is never looked at
+    far = route.copy()
+    far[0, :, 5] = 0                                     # keys 640..767 >= both... batch 0 has 700 keys: use a shorter cache
+    words = torch.from_numpy(od.pack_row(far).view(np.int32)).to(dev)
+    res = tm.tilemix_decode_int8kv(p, q.to(dev), None, k8, ks, v8, vs, words,
+                                   torch.from_numpy(np.asarray([640, 300], np.int32)).to(dev))
+    assert tm.tilemix_read_status(res["workspace"])[0] == 0

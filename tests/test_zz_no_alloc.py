@@ -13,7 +13,10 @@ def test_noalloc_entry_matches_regular_entry_twice_in_a_row():
     """Two different problems, one after the other, through the built-in workspace: each must equal the
     regular entry point's output (same kernel, so bit for bit, which is within the 2e-3 the other tests
     use), the second call must not be disturbed by what the first left in the shared workspace, and the
-    status record read back through the returned address must be clean."""
+    status record read back through the returned address must be clean.  The comparison is with the regular
+    entry point, which the other tests compare with the oracle.  torch.cuda.memory_allocated() only sees torch's
+    own allocator: that the entry point makes no allocation call of its own is a property of its source (it
+    calls cudaGetSymbolAddress, cudaMemsetAsync and the launch, nothing else), not something this test can see."""
     from paper_2608_17336_b200 import binding as b
     dev = torch.device("cuda:0")
     cases = [
@@ -57,3 +60,9 @@ def test_noalloc_entry_rejects_bad_arguments_before_launch():
     assert lib.tilemix_attention_fwd_noalloc(ctypes.byref(p), None, *args[1:], None, None, None, None) == b.ERR_NULL
     odd = b.problem(1, 2, 2, 512, 128, 64, 64)
     assert lib.tilemix_attention_fwd_noalloc(ctypes.byref(odd), *args, None, None, None, None) == b.ERR_UNSUPPORTED
+    # a stride that is not a multiple of 16 bytes: the code tilemix_attention_fwd gives, not a generic one
+    skew = b.problem(1, 2, 2, 512, 128, 128, 128)
+    skew.q_stride[0], skew.q_stride[1], skew.q_stride[2] = 2 * 512 * 132, 512 * 132, 132
+    ws = ctypes.c_void_p(0x1000)
+    assert lib.tilemix_attention_fwd(ctypes.byref(skew), *args, None, ws, 4096, None, None) == b.ERR_ALIGN
+    assert lib.tilemix_attention_fwd_noalloc(ctypes.byref(skew), *args, None, None, None, None) == b.ERR_ALIGN
