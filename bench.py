@@ -30,8 +30,8 @@ from paper_2608_17336_b200 import synth  # noqa: E402
 METRIC = "effective causal-attention TFLOP/s at 1 B200 vs INT8 fraction; % of mixed roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
-# profiles/attention_kernel_cfg3_long32k.md (8-head capture: 321.1 MB, traffic scales with the head count).
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from an ncu capture of the 8-head case of
+# the workload (321.1 MB; the traffic scales with the head count).
 NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 321.1e6 / 8}
 
 
@@ -103,14 +103,17 @@ def oracle_sample(w: synth.Workload, q, k, v, route, budget_pairs: float):
     head 0 of batch 0, as many as fit in about `budget_pairs` (query, key) pairs, plus the
     quantise and pack steps of that head.  Returns (seconds, pairs, n_rows, threads)."""
     import oracle
-    from tests import helpers as H
+
+    def np_bits(t):      # CPU half tensor -> uint16 bit patterns
+        return np.ascontiguousarray(t.contiguous().view(torch.int16).numpy()).view(np.uint16)
+
     order = np.argsort(synth.hash_uniform(w.seed + 77, 0, 0, np.arange(w.seqlen)), kind="stable")
     keep = np.cumsum(order + 1) <= budget_pairs
     keep[0] = True
     idx = np.sort(order[keep])
     rows = np.stack([np.zeros_like(idx), np.zeros_like(idx), idx], axis=1)
-    p = H.oracle_problem(w, heads=1, batch=1)
-    qb, kb, vb = (H.np_bits(t[:1, :1]) for t in (q, k, v))
+    p = oracle.Problem(1, 1, 1, w.seqlen, w.head_dim, w.tile, w.tile, w.group, mask_batch=1)
+    qb, kb, vb = (np_bits(t[:1, :1]) for t in (q, k, v))
     t0 = time.perf_counter()
     q8, qs = oracle.quantize(qb, p.bq)
     k8, ks = oracle.quantize(kb, p.bk)

@@ -9,7 +9,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("TILEMIX_LIB", os.path.join(_HERE, "libtilemix.so"))   # override: debugging builds
+LIB_PATH = os.path.join(_HERE, "libtilemix.so")
 
 OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_WORKSPACE, ERR_DEVICE_TIMEOUT = -1, -2, -3, -4, -5, -6

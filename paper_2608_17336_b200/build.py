@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.environ.get("TILEMIX_LIB", os.path.join(HERE, "libtilemix.so"))
+LIB = os.path.join(HERE, "libtilemix.so")
 SOURCES = ["api.cu", "varlen.cu", "decode.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu"]
 HEADERS = ["common.cuh", "ptx_sm100.cuh", "softmax_tile.cuh", "quant8.cuh"]
 
@@ -37,7 +37,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, f) for f in SOURCES]
-    cmd += os.environ.get("TILEMIX_NVCC_FLAGS", "").split()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -70,7 +70,7 @@ class Workload:
         return replace(self, **kw)
 
 
-# The five configurations named by the build's baseline file.
+# The five configurations the hot path is tested and measured on.
 WORKLOADS = {
     "cfg1_tiny": Workload("cfg1_tiny", 1, 1, 1024, 64, 64, 1, seed=0, routing="bernoulli",
                           int8_fraction=0.5),
