@@ -118,8 +118,10 @@ int tilemix_pack_routing_mask(const tilemix_problem_t* p, const uint8_t* route,
  *   workspace  >= tilemix_workspace_size(p) bytes, 16-byte aligned; its first 16 bytes are a
  *              status record (see tilemix_read_status) which this call clears on the stream
  *   dbg        nullable; see tilemix_debug_t
- * Requires quant_blk_q == tile_m and quant_blk_k == tile_n, 16-byte aligned bases and
- * strides, and a device of compute capability 10.0. */
+ * Requires quant_blk_q == tile_m; quant_blk_k == tile_n or tile_n / 2 (App. C "Quantization Granularity": the
+ * paper's BLK_Q = 128, BLK_K = 64 with 128 x 128 tiles; one delta_K then serves each half of a key tile; not in the
+ * on-the-fly operand mode, which quantises whole key tiles); 16-byte aligned bases and strides; a device of compute
+ * capability 10.0. */
 int tilemix_attention_fwd(const tilemix_problem_t* p, const void* q_f16, const void* k_f16,
                           const void* v_f16, const int8_t* q_i8, const int8_t* k_i8,
                           const float* q_scale, const float* k_scale,

@@ -64,7 +64,9 @@ int checked_attention(const Geometry& g, const void* q_f16, const void* k_f16, c
     const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
                           (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
     if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
+    // quantisation blocks: Q per query tile; K per key tile or per half key tile (App. C: BLK_K = BLOCK_N / 2)
+    if (g.blk_q != g.tile_m || (g.blk_k != g.tile_n && g.blk_k * 2 != g.tile_n)) return TILEMIX_ERR_UNSUPPORTED;
+    if (otf && g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;   // the on-chip quantiser works per key tile
     if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
     if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
         !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||

@@ -109,6 +109,7 @@ struct Cfg {
 struct Params {
     int B, Hq, Hk, L, G, T_m, W, nb;
     int kv_off, mask_T_m, ks_blocks;   // chunked prefill: see Geometry (0, T_m, T_m for a plain prefill)
+    int k_half_blocks;                 // 1: delta_K per half key tile (quantisation block = tile_n / 2), 0: per key tile
     int head_group;               // (batch, head) rows interleaved in the grid order (>= 1)
     int has_int8;                 // INT8 operands present
     float scale_log2;             // softmax scale * log2(e)
@@ -119,6 +120,7 @@ struct Params {
     // L = total tokens and T_m = total query-tile rows of the packed batch.
     const int32_t* vl_tok;        // [n_seqs+1] first token of each sequence
     const int32_t* vl_tile;       // [n_seqs+1] query-tile rows before each sequence
+    const int32_t* vl_blkk;       // [n_seqs+1] quantisation blocks of K before each sequence
     const int32_t* vl_item_seq;   // [total_pairs] work item -> sequence (longest rows first)
     const int32_t* vl_item_pair;  // [total_pairs] work item -> pair of query tiles of that sequence
     int n_seqs, total_pairs;
@@ -205,6 +207,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // tok0 / len: first token and length of the sequence; row0: its first row among the mask rows
     // and scale blocks; m, n below count tiles inside the sequence.
     int b, hq, pr, seq, tok0 = 0, len = prm.L, row0 = VL ? 0 : prm.kv_off, n_rows = prm.T_m;
+    int kblk0 = 0, n_kblk = prm.ks_blocks;   // first quantisation block of K of this sequence and their number
     // Order of the grid: (batch, head) rows in groups of head_group; inside a group the longest work items
     // first, and the heads of the group side by side for each item.  The host sizes the group so that its
     // K/V fits in L2 while its CTAs run; the grid then ends with the shortest items of the last group instead
@@ -235,6 +238,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
         len = prm.vl_tok[seq + 1] - tok0;
         row0 = prm.vl_tile[seq];
         n_rows = prm.vl_tile[seq + 1] - row0;
+        kblk0 = prm.vl_blkk[seq];
+        n_kblk = prm.vl_blkk[seq + 1] - kblk0;
     }
     constexpr bool varlen = VL;
     const int hk = hq / (prm.Hq / prm.Hk);
@@ -704,7 +709,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (prm.has_int8) {
                     dq = varlen ? prm.q_scale[static_cast<int64_t>(row0 + m_t) * prm.Hq + hq]
                                 : prm.q_scale[(static_cast<int64_t>(b) * prm.Hq + hq) * prm.T_m + m_t];
-                    dk_row = varlen ? prm.k_scale + static_cast<int64_t>(row0) * prm.Hk + hk
+                    dk_row = varlen ? prm.k_scale + static_cast<int64_t>(kblk0) * prm.Hk + hk
                                     : prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.ks_blocks;
                 }
             }
@@ -714,7 +719,12 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             bool ok = true;
             const int role = t ? kRoleSoftmaxB : kRoleSoftmaxA;
             bool dq_there = !OTF;   // on-the-fly mode: this tile's scale comes from the on-chip quantiser
-            float dk_next = (prm.has_int8 && !OTF) ? dk_row[0] : 0.f;
+            // delta_K of the quantisation block a step's keys lie in (App. C "Quantization Granularity": a block is a
+            // key tile or, with the paper's BLK_K = BLOCK_N / 2, one half of it -- exactly one step); the next block's
+            // scale is read ahead of its use.  A block beyond the end of a ragged sequence holds no legal key.
+            const bool k_half = prm.k_half_blocks != 0;
+            auto load_dk = [&](int blk) { return (prm.has_int8 && !OTF && blk < n_kblk) ? dk_row[blk * dk_step] : 0.f; };
+            float dk_cur = 0.f, dk_next = load_dk(0);
             float a = prm.scale_log2;
             uint32_t int8_route = 0u;
             const int n_steps = 2 * (k_t + 1);
@@ -723,14 +733,15 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             // half.  u = 2*j + h.
             for (int u = 0; u < n_steps; ++u) {
                 const int j = u >> 1, h = u & 1;
-                if (h == 0) {
-                    int8_route = (sched(j) >> t) & 1u;
+                if (h == 0) int8_route = (sched(j) >> t) & 1u;
+                if (h == 0 || k_half) {
+                    dk_cur = dk_next;
+                    dk_next = load_dk(k_half ? u + 1 : j + 1);
                     a = prm.scale_log2;
                     if (int8_route) {
-                        a *= dq * dk_next;
+                        a *= dq * dk_cur;
                         if (a == 0.f) a = 1.f;   // a zero block: every accumulator is 0 already
                     }
-                    if (!OTF && prm.has_int8 && j < k_t) dk_next = dk_row[(j + 1) * dk_step];   // next tile's scale, ahead of its use
                 }
                 const uint32_t t_sh = t_s + h * TH;
                 ok = wait_bar(cx, bar_s(t, h), j & 1, role, j, kBarS);
@@ -963,7 +974,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     int rc = get_encoder(&enc);
     if (rc) return rc;
     const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;
-    if (otf && (vl != nullptr || !(D == 128 && T == 128))) return TILEMIX_ERR_UNSUPPORTED;
+    if (otf && (vl != nullptr || !(D == 128 && T == 128) || g.blk_k != g.tile_n)) return TILEMIX_ERR_UNSUPPORTED;
     const bool has8 = !(g.flags & TILEMIX_FORCE_FP16) && (q8 != nullptr || otf);
     CUtensorMap tq, tk, tv, tq8, tk8;
     if ((rc = encode_map(enc, &tq, q, 2, g.d, g.L, g.Hq, g.B, g.qs, 64, C::kM, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
@@ -982,6 +993,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     Params prm{};
     prm.B = g.B; prm.Hq = g.Hq; prm.Hk = g.Hk; prm.L = g.L; prm.G = g.G; prm.T_m = g.T_m; prm.W = g.W;
     prm.kv_off = g.kv_off; prm.mask_T_m = g.mask_T_m; prm.ks_blocks = g.ks_blocks;
+    prm.k_half_blocks = (g.blk_k * 2 == g.tile_n) ? 1 : 0;
     {
         // heads per group: as many as keep the group's K and V (FP16; adjacent query heads of a GQA group share
         // theirs) within 72 MB of the 126 MB L2
@@ -1001,7 +1013,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     prm.lse = lse;
     prm.status = static_cast<int*>(workspace);
     if (vl != nullptr) {
-        prm.vl_tok = vl->tok; prm.vl_tile = vl->tile; prm.vl_item_seq = vl->item_seq; prm.vl_item_pair = vl->item_pair;
+        prm.vl_tok = vl->tok; prm.vl_tile = vl->tile; prm.vl_blkk = vl->blkk; prm.vl_item_seq = vl->item_seq; prm.vl_item_pair = vl->item_pair;
         prm.n_seqs = vl->n; prm.total_pairs = total_pairs;
     }
     if (dbg != nullptr && dbg->n_tiles > 0) {

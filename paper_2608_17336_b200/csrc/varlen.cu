@@ -188,7 +188,7 @@ int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varle
     const bool shape_ok = (g.d == 128 && g.tile_m == 128 && g.tile_n == 128) ||
                           (g.d == 64 && g.tile_m == 64 && g.tile_n == 64);
     if (!shape_ok) return TILEMIX_ERR_UNSUPPORTED;
-    if (g.blk_q != g.tile_m || g.blk_k != g.tile_n) return TILEMIX_ERR_UNSUPPORTED;
+    if (g.blk_q != g.tile_m || (g.blk_k != g.tile_n && g.blk_k * 2 != g.tile_n)) return TILEMIX_ERR_UNSUPPORTED;
     if (g.T_n > 2048) return TILEMIX_ERR_UNSUPPORTED;   // schedule table of the kernel
     if (!aligned16(q_f16) || !aligned16(k_f16) || !aligned16(v_f16) || !aligned16(out_f16) ||
         !aligned16(workspace) || (!force16 && (!aligned16(q_i8) || !aligned16(k_i8))) ||
