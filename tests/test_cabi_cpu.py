@@ -65,7 +65,10 @@ def test_host_side_validation_without_gpu(lib):
         ctypes.byref(p), *_args(3), ctypes.c_void_p(q8) if q8 else None, *_args(5), None, ctypes.c_void_p(0x1000), ws, None, None)
     assert att(b.problem(1, 2, 2, 1024, 128, 64, 64)) == b.ERR_UNSUPPORTED
     assert att(b.problem(1, 2, 2, 1024, 96, 128, 128)) == b.ERR_UNSUPPORTED
-    assert att(b.problem(1, 2, 2, 1024, 128, 128, 128, quant_blk_k=64)) == b.ERR_UNSUPPORTED
+    # quantisation blocks: K per key tile or per half key tile, Q per query tile; the on-the-fly mode per tile only
+    assert att(b.problem(1, 2, 2, 1024, 128, 128, 128, quant_blk_k=32)) == b.ERR_UNSUPPORTED
+    assert att(b.problem(1, 2, 2, 1024, 128, 128, 128, quant_blk_q=64)) == b.ERR_UNSUPPORTED
+    assert att(b.problem(1, 2, 2, 1024, 128, 128, 128, quant_blk_k=64, flags=b.QUANT_ON_THE_FLY)) == b.ERR_UNSUPPORTED
     assert att(good, ws=8) == b.ERR_WORKSPACE
     assert att(good, q8=0) == b.ERR_NULL
     assert att(good, q8=0x1001) == b.ERR_ALIGN
