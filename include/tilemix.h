@@ -322,6 +322,16 @@ int tilemix_read_status(const void* workspace, int32_t out[4], void* stream);
 const char* tilemix_status_string(int code);
 /* Number of kernels this library has launched since it was loaded (all entry points). */
 uint64_t tilemix_launch_count(void);
+/* Testing aid for the bounded waits (the paper has no counterpart).  Every wait inside the kernels is bounded: when
+ * one runs out the CTA records {TILEMIX_ERR_DEVICE_TIMEOUT, role, tile, barrier} in the status record, every role
+ * stops, what is in flight is waited for, and the kernel RETURNS -- nothing faults and nothing spins for ever.  This
+ * switch, process-wide and read at launch time, lets a test see that path run:
+ *   which = 1  the attention kernel's producer leaves out the copies of operand bundle 1 (V of key tile 0 and K of key
+ *              tile 1) of every CTA, so an MMA issuer's wait for that bundle runs out after wait_limit_ns
+ *   which = 2  the decode step's producer leaves out the second tile of every split
+ *   which = 0  normal operation, limit back to the default of 2 s (wait_limit_ns is ignored)
+ * Returns TILEMIX_OK or TILEMIX_ERR_SHAPE. */
+int tilemix_test_drop_copy(int which, uint64_t wait_limit_ns);
 
 #ifdef __cplusplus
 }

@@ -25,6 +25,7 @@ EXPORTS = (
     "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
     "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
     "tilemix_decode_workspace_size", "tilemix_decode_int8kv", "tilemix_attention_fwd_chunk",
+    "tilemix_test_drop_copy",
 )
 
 
@@ -106,6 +107,7 @@ def lib() -> ctypes.CDLL:
         L.tilemix_status_string.argtypes = [i32]
         L.tilemix_status_string.restype = ctypes.c_char_p
         L.tilemix_launch_count.restype = ctypes.c_uint64
+        L.tilemix_test_drop_copy.argtypes = [i32, ctypes.c_uint64]
         dp = ctypes.POINTER(DecodeStruct)
         L.tilemix_decode_workspace_size.argtypes = [dp]
         L.tilemix_decode_workspace_size.restype = ctypes.c_size_t
@@ -254,6 +256,11 @@ def tilemix_workspace_size(p): return int(lib().tilemix_workspace_size(ctypes.by
 def tilemix_scratch_bytes(p): return int(lib().tilemix_scratch_bytes(ctypes.byref(p)))
 def tilemix_mask_words_per_row(seqlen, tile_n, group): return int(lib().tilemix_mask_words_per_row(seqlen, tile_n, group))
 def tilemix_launch_count(): return int(lib().tilemix_launch_count())
+
+
+def tilemix_test_drop_copy(which: int, wait_limit_ns: int = 0):
+    """Testing aid of the bounded waits (see tilemix.h); which = 0 switches it off."""
+    _check(lib().tilemix_test_drop_copy(which, wait_limit_ns), "tilemix_test_drop_copy")
 
 
 # ------------------------------------------------------------------ variable-length batches

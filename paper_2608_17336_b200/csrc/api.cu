@@ -9,6 +9,8 @@
 namespace tilemix {
 
 std::atomic<uint64_t> g_launch_count{0};
+std::atomic<int> g_test_drop{0};
+std::atomic<uint64_t> g_wait_limit_ns{kDefaultWaitLimitNs};
 
 namespace {
 
@@ -385,5 +387,12 @@ const char* tilemix_status_string(int code) {
 }
 
 uint64_t tilemix_launch_count(void) { return g_launch_count.load(); }
+
+int tilemix_test_drop_copy(int which, uint64_t wait_limit_ns) {
+    if (which < 0 || which > 2) return TILEMIX_ERR_SHAPE;
+    g_test_drop.store(which);
+    g_wait_limit_ns.store(which == 0 || wait_limit_ns == 0 ? kDefaultWaitLimitNs : wait_limit_ns);
+    return TILEMIX_OK;
+}
 
 }  // extern "C"

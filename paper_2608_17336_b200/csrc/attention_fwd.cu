@@ -55,7 +55,6 @@ constexpr int kRing = 8;
 constexpr int kBundles = 4;        // operand bundles in flight at most (each has a "landed" and a "consumed" barrier)
 constexpr int kWorkspaceClearBytes = 4096;  // status record
 constexpr int kMaxTiles = 2048;           // key tiles per row the shared-memory schedule table holds
-constexpr uint64_t kTimeoutNs = 2000000000ull;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 // Lazy running maximum.  P = 2^(score - m) is handed to the tensor pipe in FP16 (largest finite value just
@@ -110,6 +109,8 @@ struct Params {
     int B, Hq, Hk, L, G, T_m, W, nb;
     int kv_off, mask_T_m, ks_blocks;   // chunked prefill: see Geometry (0, T_m, T_m for a plain prefill)
     int k_half_blocks;                 // 1: delta_K per half key tile (quantisation block = tile_n / 2), 0: per key tile
+    unsigned long long wait_limit_ns;  // limit of every bounded wait
+    int test_drop_bundle;              // testing aid: the producer leaves out the copies of this operand bundle (-1: none)
     int head_group;               // (batch, head) rows interleaved in the grid order (>= 1)
     int has_int8;                 // INT8 operands present
     float scale_log2;             // softmax scale * log2(e)
@@ -137,6 +138,7 @@ struct Params {
 struct Ctx {
     volatile int* abort_flag;
     int* status;
+    unsigned long long wait_limit_ns;
 };
 
 __device__ __forceinline__ void record_timeout(const Ctx& cx, int role, int tile, int which) {
@@ -157,7 +159,7 @@ __device__ __forceinline__ bool wait_bar(const Ctx& cx, uint32_t bar, uint32_t p
     while (!ptx::mbar_try_wait(bar, parity)) {
         if ((++it & 127u) == 0u) {
             if (*cx.abort_flag) return false;
-            if (ptx::globaltimer_ns() - t0 > kTimeoutNs) {
+            if (ptx::globaltimer_ns() - t0 > cx.wait_limit_ns) {
                 record_timeout(cx, role, tile, which);
                 return false;
             }
@@ -277,7 +279,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     volatile float* otf_dk = reinterpret_cast<volatile float*>(misc + 4);
     volatile float* otf_dq = reinterpret_cast<volatile float*>(misc + 12);
     uint32_t* sched_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
-    Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status};
+    Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status, prm.wait_limit_ns};
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar_q(0), 1);
@@ -492,6 +494,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 }
             };
             int armed = 0;                          // bundles whose copies have been issued
+            int dropped = -1;                       // (testing aid) the bundle that was left out
             for (int n = 0; n <= nkv && ok; ++n) {
                 // bundle n: V of key tile n - 1 (n >= 1) and the K copies of key tile n (n < nkv)
                 const uint32_t e = n < nkv ? sched(n) : 0u;
@@ -505,6 +508,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (e & 4u) { s16 = ring.take(C::kHalves); (make8 ? raw_bytes : bytes) += C::kHalves * C::kChunk; }
                 if (e & 8u) { s8 = ring.take(1); if (!OTF) bytes += C::kK8Bytes; }
                 if (bytes == 0u && raw_bytes == 0u) break;             // nothing after the last V
+                if (n == prm.test_drop_bundle) {   // testing aid: this bundle never lands, an issuer's bounded wait runs out
+                    dropped = n;
+                    continue;
+                }
                 if (n >= kBundles) wait_consumed(n - kBundles, n);     // its barriers are free again
                 // the barrier is armed for the whole bundle first; every operand is then copied as soon as
                 // its own chunks are free, so a V tile does not wait for the room of the K tile behind it
@@ -550,6 +557,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             if (!ok || *cx.abort_flag) {
                 // let copies that are still in flight land before the CTA's memory is released
                 for (int n = armed > kBundles ? armed - kBundles : 0; n < armed; ++n) {
+                    if (n == dropped) continue;
                     for (int it = 0; it < (1 << 20); ++it)
                         if (ptx::mbar_try_wait(bar_full(n % kBundles), (n / kBundles) & 1)) break;
                     if (OTF && n < nkv)
@@ -994,6 +1002,8 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     prm.B = g.B; prm.Hq = g.Hq; prm.Hk = g.Hk; prm.L = g.L; prm.G = g.G; prm.T_m = g.T_m; prm.W = g.W;
     prm.kv_off = g.kv_off; prm.mask_T_m = g.mask_T_m; prm.ks_blocks = g.ks_blocks;
     prm.k_half_blocks = (g.blk_k * 2 == g.tile_n) ? 1 : 0;
+    prm.wait_limit_ns = g_wait_limit_ns.load();
+    prm.test_drop_bundle = g_test_drop.load() == 1 ? 1 : -1;
     {
         // heads per group: as many as keep the group's K and V (FP16; adjacent query heads of a GQA group share
         // theirs) within 72 MB of the 126 MB L2

@@ -36,12 +36,13 @@ struct DecodeParams {
     int8_t* q8_out;
     float* qs_out;
     int* status;     // 4 ints at the start of the workspace (same record as the attention kernel's)
+    unsigned long long wait_limit_ns;   // limit of the bounded waits
+    int test_drop_tile;                 // testing aid: the producer leaves out the copies of this tile of every split (-1: none)
 };
 
 constexpr int kStages = 2;    // ring of key/value tiles in shared memory when FP16 keys may be read ...
 constexpr int kStagesInt8 = 3;   // ... and when there is no FP16 key cache (a stage is a third smaller)
 constexpr int kChunk = 128;   // keys per kernel tile when tile_n allows it (64-key tiles with deeper rings were slower)
-constexpr uint64_t kTimeoutNs = 2000000000ull;
 
 template <int D, int T>
 struct Stage {
@@ -179,7 +180,7 @@ decode_kernel(const DecodeParams prm) {
         while (!ptx::mbar_try_wait(addr, parity)) {
             if ((++spins & 63u) == 0u) {
                 if (*reinterpret_cast<volatile int*>(&abort_flag)) return false;
-                if (ptx::globaltimer_ns() - start > kTimeoutNs) {
+                if (ptx::globaltimer_ns() - start > prm.wait_limit_ns) {
                     *reinterpret_cast<volatile int*>(&abort_flag) = 1;
                     return false;
                 }
@@ -219,8 +220,10 @@ decode_kernel(const DecodeParams prm) {
     const int8_t* k8 = prm.k8 + row_base * D;
     const int8_t* v8 = prm.v8 + row_base * D;
     const __half* k16 = prm.k16 != nullptr ? prm.k16 + row_base * D : nullptr;
+    int last_produced = -1;   // (producer lane) the last tile whose copies were started
     auto produce = [&](int tile) -> bool {
         const int it = tile - t0, stage = it % n_stages;
+        if (it == prm.test_drop_tile) return true;   // testing aid: this tile never lands, the consumers' bounded wait runs out
         // the first pass over the ring finds every stage free
         if (it >= n_stages && !wait_ring(&empty_bar[stage], ((it / n_stages) - 1) & 1)) return false;
         const uint32_t rows = static_cast<uint32_t>(min(T, len - tile * T));   // only rows that exist
@@ -232,6 +235,7 @@ decode_kernel(const DecodeParams prm) {
         if (int8) ptx::bulk_load_1d(dst, k8 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
         else ptx::bulk_load_1d(dst, k16 + static_cast<int64_t>(tile) * T * D, kbytes, bar);
         ptx::bulk_load_1d(dst + k_slot, v8 + static_cast<int64_t>(tile) * T * D, rows * D, bar);
+        last_produced = tile;
         return true;
     };
     const bool producer = warp == kConsumerWarps - 1 && lane == 0;
@@ -384,6 +388,15 @@ decode_kernel(const DecodeParams prm) {
     if (*reinterpret_cast<volatile int*>(&abort_flag)) {
         if (tid == 0 && atomicCAS(&prm.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
             prm.status[1] = 16; prm.status[2] = t0; prm.status[3] = 0;
+        }
+        // the copies still in flight land before this CTA's shared memory is given back (each stage's latest one)
+        if (producer) {
+            for (int tile = max(t0, last_produced - n_stages + 1); tile <= last_produced; ++tile) {
+                const int it = tile - t0;
+                if (it == prm.test_drop_tile) continue;
+                for (int spin = 0; spin < (1 << 16); ++spin)
+                    if (ptx::mbar_try_wait(ptx::smem_u32(&full_bar[it % n_stages]), (it / n_stages) & 1)) break;
+            }
         }
         return;
     }
@@ -573,6 +586,8 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     prm.k8 = k_i8; prm.k_scale = k_scale; prm.v8 = v_i8; prm.v_scale = v_scale;
     prm.words = mask_words;
     prm.status = static_cast<int*>(workspace);
+    prm.wait_limit_ns = g_wait_limit_ns.load();
+    prm.test_drop_tile = g_test_drop.load() == 2 ? 1 : -1;
     int32_t* len_ws = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kDecodeStatusBytes);
     prm.cache_len = len_ws;
     uint8_t* ws = static_cast<uint8_t*>(workspace) + kDecodeStatusBytes + decode_len_bytes(p->batch);

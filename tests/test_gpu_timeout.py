@@ -1,0 +1,73 @@
+"""The bounded waits of the kernels, seen running out -- without a fault, a trap or an endless loop.
+
+A testing switch of the library makes a producer leave out one copy, so that the wait for it runs out after a few
+milliseconds; the CTA then records a status, every role stops, what is in flight is waited for and the kernel
+returns.  The tests read the status record and then use the same workspace for a normal call."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decode as od
+from paper_2608_17336_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+ROLE_MMA, BAR_RING_FULL = 3, 1       # the role / barrier numbers of the attention kernel's status record
+
+
+@pytest.fixture
+def drop():
+    from paper_2608_17336_b200 import binding as tm
+    yield tm.tilemix_test_drop_copy
+    tm.tilemix_test_drop_copy(0)        # always back to normal operation
+
+
+def test_attention_wait_runs_out_and_the_kernel_returns(drop):
+    from paper_2608_17336_b200 import binding as tm
+    w = synth.Workload("timeout", 1, 2, 1024, 128, 128, 1, seed=91, routing="bernoulli", int8_fraction=0.5)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(w))
+    route = torch.from_numpy(synth.make_route(w)).to(DEV)
+    p = H.gpu_problem(w)
+    q8, k8, qs, ks = tm.tilemix_quantize_qk(p, q, k)
+    words, _ = tm.tilemix_pack_routing_mask(p, route, False)
+    good = tm.tilemix_attention_fwd(p, q, k, v, q8, k8, qs, ks, words)
+    assert tm.tilemix_read_status(good["workspace"])[0] == 0
+    ws = good["workspace"]
+    drop(1, 2_000_000)                  # the wait for operand bundle 1 runs out after 2 ms
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    bad = tm.tilemix_attention_fwd(p, q, k, v, q8, k8, qs, ks, words, workspace=ws)
+    t1.record()
+    code, rec = tm.tilemix_read_status(bad["workspace"])
+    assert code == tm.ERR_DEVICE_TIMEOUT
+    assert rec[1] == ROLE_MMA and rec[2] == 1 and rec[3] == BAR_RING_FULL, rec
+    assert t0.elapsed_time(t1) < 500.0            # it returned after the short limit, not after the default 2 s
+    drop(0)
+    again = tm.tilemix_attention_fwd(p, q, k, v, q8, k8, qs, ks, words, workspace=ws)
+    assert tm.tilemix_read_status(again["workspace"])[0] == 0
+    assert torch.equal(again["out"], good["out"])
+
+
+def test_decode_wait_runs_out_and_the_kernel_returns(drop):
+    from paper_2608_17336_b200 import binding as tm
+    B, Hq, Hk, L, d, tile = 2, 4, 2, 1500, 128, 128
+    gen = torch.Generator(device="cpu").manual_seed(92)
+    q = torch.randn((B, Hq, d), generator=gen).half().to(DEV)
+    k = torch.randn((B, Hk, L, d), generator=gen).half().to(DEV)
+    v = torch.randn((B, Hk, L, d), generator=gen).half().to(DEV)
+    k8, v8, ks, vs = tm.tilemix_quantize_qk(tm.problem(B, Hk, Hk, L, d, tile, tile), k, v)
+    route = (np.random.default_rng(1).random((1, Hk, -(-L // tile))) < 0.5).astype(np.uint8)
+    words = torch.from_numpy(od.pack_row(route).view(np.int32)).to(DEV)
+    lens = torch.from_numpy(np.asarray([1500, 900], np.int32)).to(DEV)
+    p = tm.decode_problem(B, Hq, Hk, d, L, tile, 1, n_splits=2)      # every split has several tiles
+    good = tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words, lens)
+    assert tm.tilemix_read_status(good["workspace"])[0] == 0
+    drop(2, 2_000_000)
+    bad = tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words, lens, workspace=good["workspace"])
+    code, rec = tm.tilemix_read_status(bad["workspace"])
+    assert code == tm.ERR_DEVICE_TIMEOUT, rec
+    drop(0)
+    again = tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words, lens, workspace=good["workspace"])
+    assert tm.tilemix_read_status(again["workspace"])[0] == 0
+    assert torch.equal(again["out"], good["out"])
