@@ -322,6 +322,13 @@ int tilemix_read_status(const void* workspace, int32_t out[4], void* stream);
 const char* tilemix_status_string(int code);
 /* Number of kernels this library has launched since it was loaded (all entry points). */
 uint64_t tilemix_launch_count(void);
+/* Measurement aid (the paper has no counterpart): the issue rate of the tensor pipe for the instruction shape the
+ * fused kernel's full score tile uses, the denominator of its roofline measured on the same GPU in the same run.  One
+ * CTA per SM issues n_mma back-to-back tcgen05.mma M128 N128 (K16 kind::f16 if int8 == 0, K32 kind::i8 otherwise)
+ * with both operands in shared memory, into one accumulator, and returns when they have retired.  Time the call with
+ * events on `stream`: operations = *n_ctas * n_mma * 2*128*128*K.  workspace: >= 16 device bytes, receives a status
+ * record (tilemix_read_status).  Returns TILEMIX_OK, TILEMIX_ERR_SHAPE or a CUDA error. */
+int tilemix_tensor_peak_probe(int int8, int n_mma, int* n_ctas, void* workspace, void* stream);
 /* Testing aid for the bounded waits (the paper has no counterpart).  Every wait inside the kernels is bounded: when
  * one runs out the CTA records {TILEMIX_ERR_DEVICE_TIMEOUT, role, tile, barrier} in the status record, every role
  * stops, what is in flight is waited for, and the kernel RETURNS -- nothing faults and nothing spins for ever.  This

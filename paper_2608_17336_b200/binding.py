@@ -25,7 +25,7 @@ EXPORTS = (
     "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
     "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
     "tilemix_decode_workspace_size", "tilemix_decode_int8kv", "tilemix_attention_fwd_chunk",
-    "tilemix_test_drop_copy",
+    "tilemix_test_drop_copy", "tilemix_tensor_peak_probe",
 )
 
 
@@ -108,6 +108,7 @@ def lib() -> ctypes.CDLL:
         L.tilemix_status_string.restype = ctypes.c_char_p
         L.tilemix_launch_count.restype = ctypes.c_uint64
         L.tilemix_test_drop_copy.argtypes = [i32, ctypes.c_uint64]
+        L.tilemix_tensor_peak_probe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_int), vp, vp]
         dp = ctypes.POINTER(DecodeStruct)
         L.tilemix_decode_workspace_size.argtypes = [dp]
         L.tilemix_decode_workspace_size.restype = ctypes.c_size_t
@@ -256,6 +257,13 @@ def tilemix_workspace_size(p): return int(lib().tilemix_workspace_size(ctypes.by
 def tilemix_scratch_bytes(p): return int(lib().tilemix_scratch_bytes(ctypes.byref(p)))
 def tilemix_mask_words_per_row(seqlen, tile_n, group): return int(lib().tilemix_mask_words_per_row(seqlen, tile_n, group))
 def tilemix_launch_count(): return int(lib().tilemix_launch_count())
+
+
+def tilemix_tensor_peak_probe(int8: bool, n_mma: int, workspace) -> int:
+    """Enqueues the tensor-pipe issue-rate probe on the current stream; returns the number of CTAs (time it with events)."""
+    n = ctypes.c_int(0)
+    _check(lib().tilemix_tensor_peak_probe(1 if int8 else 0, n_mma, ctypes.byref(n), _ptr(workspace), _stream()), "tilemix_tensor_peak_probe")
+    return n.value
 
 
 def tilemix_test_drop_copy(which: int, wait_limit_ns: int = 0):

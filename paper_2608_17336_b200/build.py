@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtilemix.so")
-SOURCES = ["api.cu", "varlen.cu", "decode.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu"]
+SOURCES = ["api.cu", "varlen.cu", "decode.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu", "peak_probe.cu"]
 HEADERS = ["common.cuh", "ptx_sm100.cuh", "softmax_tile.cuh", "quant8.cuh"]
 
 
