@@ -265,7 +265,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     // per query tile t and half h of the score tile: "S half ready", "P half ready"; per tile: "PV retired"
     auto bar_s = [&](int t, int h) { return bar0 + 8u * (2 + 2 * kRing + 2 * t + h); };
     auto bar_p = [&](int t, int h) { return bar0 + 8u * (6 + 2 * kRing + 2 * t + h); };
-    auto bar_pv = [&](int t) { return bar0 + 8u * (10 + 2 * kRing + t); };   // every PV of tile t
+    auto bar_pv = [&](int t) { return bar0 + 8u * (10 + 2 * kRing + t); };   // the last-but-one PV of tile t
     auto bar_o = [&](int t) { return bar0 + 8u * (12 + 2 * kRing + t); };    // the last PV of tile t
     const uint32_t bar_drain = bar0 + 8u * (14 + 2 * kRing);
     // on-the-fly mode: "FP16 K tile of bundle i landed and its INT8 chunk is free" (producer -> quantiser),
@@ -678,7 +678,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         if (!wait_bar(cx, bar_p(t, h), j & 1, kRoleMma, j, kBarP)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
                         issue_pv(t, h, sv, (j > 0 || h > 0) ? 1u : 0u);
-                        ptx::mma_commit(bar_pv(t));
+                        if (j == m_t && h == 0) ptx::mma_commit(bar_pv(t));   // the last-but-one PV (a rescale in the last step waits for it)
                         if (j == m_t && h == 1) ptx::mma_commit(bar_o(t));
                         if (more) {
                             issue_qk(t, h, r_next, k16, k8);
@@ -866,12 +866,14 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 z[0] += sum[0];
                 z[1] += sum[1];
 
-                if (u > 0 && __any_sync(0xffffffffu, grow)) {
+                if (redo && u > 0 && __any_sync(0xffffffffu, grow)) {
                     // O~ *= alpha.  The PV of the previous step may still be accumulating into O~: wait
                     // until it has retired (the PV of this step is not issued before P arrives below).
-                    // The S half seen above was issued behind PV(u-2), so that barrier is in phase u-1
-                    // or u and its parity is unambiguous.
-                    ok = wait_bar(cx, bar_pv(t), (u - 1) & 1, role, j, kBarPV);
+                    // The issuer puts the QK^T of step u+1 behind PV(u-1) and commits both to "S(u+1) ready",
+                    // so that barrier -- the one the next step waits on anyway -- says PV(u-1) has retired; the
+                    // last step has no successor and waits on the commit behind the last-but-one PV instead.
+                    if (u + 1 < n_steps) ok = wait_bar(cx, bar_s(t, h ^ 1), ((u + 1) >> 1) & 1, role, j, kBarS);
+                    else ok = wait_bar(cx, bar_pv(t), 0, role, j, kBarPV);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
