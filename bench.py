@@ -31,8 +31,8 @@ METRIC = "effective causal-attention TFLOP/s at 1 B200 vs INT8 fraction; % of mi
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from an ncu capture of the 8-head case of
-# the workload (321.1 MB; the traffic scales with the head count).
-NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 321.1e6 / 8}
+# the workload (488.4 MB; the traffic scales with the head count).
+NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 488.4e6 / 8}
 
 
 def effective_flops(w: synth.Workload) -> float:
@@ -508,15 +508,15 @@ def main():
             words_s, _ = tm.tilemix_pack_routing_mask(p, torch.from_numpy(synth.make_route(ws)).to(dev), False)
             whs = words_s.cpu().numpy().view(np.uint32)
             f8s = float(((whs[:, :, mm, gg >> 5] >> (gg & 31).astype(np.uint32)) & 1).mean())
-            for _ in range(2):
+            for _ in range(3):
                 tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words_s, out=out, workspace=work)
-            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            s0.record(stream)
-            for _ in range(5):
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(7)]
+            for s0, s1 in evs:
+                s0.record(stream)
                 tm.tilemix_attention_fwd(p, qd, kd, vd, q8, k8, qs, ks, words_s, out=out, workspace=work)
-            s1.record(stream)
+                s1.record(stream)
             torch.cuda.synchronize()
-            ms = s0.elapsed_time(s1) / 5
+            ms = statistics.median(s0.elapsed_time(s1) for s0, s1 in evs)   # median of 7 launches
             pk = p16 / (1.0 - f8s * (1.0 - 1.0 / INT8_OVER_FP16) / 2.0)
             sweep.append({"int8_tiles": round(f8s, 4), "attention_ms": round(ms, 4),
                           "tflops": round(F / (ms * 1e-3) / 1e12, 1), "frac": round(F / (ms * 1e-3) / 1e12 / pk, 4)})
