@@ -12,8 +12,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtilemix.so")
-SOURCES = ["api.cu", "varlen.cu", "decode.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu", "peak_probe.cu"]
-HEADERS = ["common.cuh", "ptx_sm100.cuh", "softmax_tile.cuh", "quant8.cuh"]
+SOURCES = ["api.cu", "varlen.cu", "decode.cu", "decode_umma.cu", "quantize.cu", "pack_mask.cu", "attention_fwd.cu", "peak_probe.cu"]
+HEADERS = ["common.cuh", "decode.cuh", "ptx_sm100.cuh", "softmax_tile.cuh", "quant8.cuh"]
 
 
 def _nvcc() -> str:

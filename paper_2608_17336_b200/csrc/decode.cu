@@ -9,6 +9,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "decode.cuh"
 #include "ptx_sm100.cuh"
 
 namespace tilemix {
@@ -18,27 +19,6 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-struct DecodeParams {
-    int B, Hq, Hk, max_len, G, nb, W, n_splits, n_blk;
-    int tile_n;      // tokens per scale block and per routing key tile (a multiple of the kernel's chunk)
-    float scale_log2;
-    const __half* q;
-    const __half* k16;
-    const int8_t* k8;
-    const float* k_scale;
-    const int8_t* v8;
-    const float* v_scale;
-    const uint32_t* words;
-    const int32_t* cache_len;
-    float* o_part;   // [B, Hq, n_splits, D]
-    float* m_part;   // [B, Hq, n_splits]
-    float* z_part;
-    int8_t* q8_out;
-    float* qs_out;
-    int* status;     // 4 ints at the start of the workspace (same record as the attention kernel's)
-    unsigned long long wait_limit_ns;   // limit of the bounded waits
-    int test_drop_tile;                 // testing aid: the producer leaves out the copies of this tile of every split (-1: none)
-};
 
 constexpr int kStages = 2;    // ring of key/value tiles in shared memory when FP16 keys may be read ...
 constexpr int kStagesInt8 = 3;   // ... and when there is no FP16 key cache (a stage is a third smaller)
@@ -450,6 +430,7 @@ __global__ void __launch_bounds__(D)
 decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ m_part,
                     const float* __restrict__ z_part, int n_splits, __half* __restrict__ out,
                     float* __restrict__ lse) {
+    ptx::griddep_wait();   // (when launched as a programmatic dependent of the step kernel)
     const int64_t row = blockIdx.x;
     const int e = threadIdx.x;
     float m = -INFINITY;
@@ -503,6 +484,7 @@ constexpr size_t kDecodeStatusBytes = 256;   // status record of the bounded wai
 // workspace (they live on the device, so the host cannot check them; the step itself reads the copy).
 __global__ void decode_prepare_kernel(const int32_t* __restrict__ cache_len, int B, int max_len, int* status,
                                       int32_t* __restrict__ len_out) {
+    ptx::griddep_launch_dependents();   // the step kernel may set itself up meanwhile; it waits before it reads these
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < 4) status[i] = 0;
     if (i < B) len_out[i] = min(max(cache_len[i], 0), max_len);
@@ -605,7 +587,22 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     if (pe != cudaSuccess) return static_cast<int>(pe);
     // keys are streamed and processed one routing tile at a time (64-key chunks with a deeper ring
     // were slower: the per-chunk barriers cost more than the extra bytes in flight gain)
-    if (p->head_dim == 128 && p->tile_n == 128) return launch_r<128, kChunk>(R, prm, out, lse, s);
+    if (p->head_dim == 128 && p->tile_n == 128) {
+        // the tcgen05 form of the step (decode_umma.cu), then the same merge
+        rc = launch_decode_umma(R, prm, s);
+        if (rc) return rc;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(prm.B * prm.Hq); cfg.blockDim = dim3(128); cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const cudaError_t me = cudaLaunchKernelEx(&cfg, decode_merge_kernel<128>, static_cast<const float*>(prm.o_part),
+                                                  static_cast<const float*>(prm.m_part), static_cast<const float*>(prm.z_part),
+                                                  prm.n_splits, out, lse);
+        g_launch_count.fetch_add(1);
+        return static_cast<int>(me);
+    }
     if (p->head_dim == 128 && p->tile_n == 64) return launch_r<128, 64>(R, prm, out, lse, s);
     if (p->head_dim == 64 && p->tile_n == 128) return launch_r<64, kChunk>(R, prm, out, lse, s);
     if (p->head_dim == 64 && p->tile_n == 64) return launch_r<64, 64>(R, prm, out, lse, s);
