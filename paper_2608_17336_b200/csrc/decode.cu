@@ -494,6 +494,7 @@ size_t decode_len_bytes(int B) { return (static_cast<size_t>(B) * sizeof(int32_t
 
 struct DecodeGeometry {
     int n_blk, T_mask, W, n_splits;
+    int n_parts;            // partial results per query head in the workspace (the tcgen05 form writes two per split)
     size_t o_bytes, mz_bytes;
 };
 
@@ -524,7 +525,8 @@ int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     if (splits > g->n_blk) splits = g->n_blk;
     if (splits > 65535) return TILEMIX_ERR_UNSUPPORTED;
     g->n_splits = splits;
-    const size_t rows = static_cast<size_t>(p->batch) * p->heads_q * splits;
+    g->n_parts = (p->head_dim == 128 && p->tile_n == 128) ? 2 * splits : splits;
+    const size_t rows = static_cast<size_t>(p->batch) * p->heads_q * g->n_parts;
     g->o_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
     g->mz_bytes = (rows * sizeof(float) + 255) / 256 * 256;
     return TILEMIX_OK;
@@ -599,7 +601,7 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
         cfg.attrs = attr; cfg.numAttrs = 1;
         const cudaError_t me = cudaLaunchKernelEx(&cfg, decode_merge_kernel<128>, static_cast<const float*>(prm.o_part),
                                                   static_cast<const float*>(prm.m_part), static_cast<const float*>(prm.z_part),
-                                                  prm.n_splits, out, lse);
+                                                  g.n_parts, out, lse);
         g_launch_count.fetch_add(1);
         return static_cast<int>(me);
     }

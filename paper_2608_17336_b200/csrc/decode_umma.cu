@@ -52,13 +52,28 @@ constexpr int kOffMeta = kOffV16 + 2 * kVBytes;
 constexpr int kOffSmall = kOffMeta + kMetaTiles * 8;
 static_assert(kOffRing % 1024 == 0 && kOffV16 % 1024 == 0, "swizzled tiles start on 1 KB boundaries");
 
-constexpr int kSoftmaxWarps = 4, kConvWarps = 16;
+// Two independent softmax streams of four warps each: stream g takes the steps (pairs of key tiles) j = g, g + 2, ...
+// with its own running maximum, row sums and O accumulator, and ends as its own partial result -- to the merge
+// kernel a CTA is two splits.  A stream's step is a chain of waits and short dependent instruction runs
+// (~2600 clk); two of them in flight hide that latency.
+constexpr int kStreams = 2, kStreamWarps = 4, kSoftmaxWarps = kStreams * kStreamWarps, kConvWarps = 16;
 constexpr int kConvWarp0 = kSoftmaxWarps, kProducerWarp = kConvWarp0 + kConvWarps;
 constexpr int kQkWarp = kProducerWarp + 1, kPvWarp = kQkWarp + 1;
-constexpr int kThreads = (kPvWarp + 1) * 32;
+constexpr int kThreads = (kPvWarp + 2) * 32;   // one idle warp completes the last group of four (setmaxnreg)
 constexpr int kConvThreads = kConvWarps * 32;
-constexpr int kTmemCols = 256;            // S^T: four buffers of 16 columns from column 0; O: columns 128..255
+constexpr int kTmemCols = 512;            // S^T: four buffers of 16 columns from column 0; O of stream g: 128 + 128 g
 constexpr uint32_t kColO = 128;
+// Registers: the block is launched with kLaunchRegs per thread; the conversion warps, which hold kVDepth tiles of V8
+// in flight, take more, the others hand theirs back.  The split must add up to the launch allotment exactly
+// (setmaxnreg.inc waits for registers that other warps release: a split above the allotment would wait for ever;
+// the host refuses to launch when the compiler planned for fewer registers than kLaunchRegs).
+constexpr int kLaunchRegs = 72, kRegsCtl = 40;
+template <int R> struct Regs {
+    static constexpr int kConv = R == 8 ? 80 : 88, kSoft = R == 8 ? 72 : 56;
+    static_assert(kConvThreads * kConv + kSoftmaxWarps * 32 * kSoft + 4 * 32 * kRegsCtl == kThreads * kLaunchRegs,
+                  "setmaxnreg split");
+};
+static_assert(kThreads == 896 && kThreads % 128 == 0, "warp groups of four");
 constexpr float kMoveAbove = 8.f;         // m moves when a step's maximum exceeds it by more than 2^8
 
 struct Small {
@@ -66,10 +81,10 @@ struct Small {
     uint64_t s_ready[2], s_free[2], p_ready[2], xchg[2];      // per pair buffer
     uint64_t v_ready[2], pv_done[2];                          // per V16 buffer (tile parity)
     uint64_t pv_pair[2];                                      // per pair buffer: the PVs of a step have retired
-    uint64_t zbar, drain_qk, drain_pv;
+    uint64_t zbar[kStreams], drain_qk, drain_pv;
     uint32_t slot_info[kSlots];           // ring units of the key tile in a slot: byte 0, second FP16 slab: byte 1
-    float warp_max[2][kSoftmaxWarps][8];
-    float zsum[kSoftmaxWarps][8];
+    float warp_max[kStreams][kStreamWarps][8];
+    float zsum[kStreams][kStreamWarps][8];
     float dq[8];
     uint32_t tmem_base;
     int abort_flag;
@@ -101,14 +116,14 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.s_ready[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.s_free[i]), kSoftmaxWarps * 32);
-            ptx::mbar_init(ptx::smem_u32(&sh.p_ready[i]), kSoftmaxWarps * 32);
-            ptx::mbar_init(ptx::smem_u32(&sh.xchg[i]), kSoftmaxWarps);
+            ptx::mbar_init(ptx::smem_u32(&sh.s_free[i]), kStreamWarps * 32);
+            ptx::mbar_init(ptx::smem_u32(&sh.p_ready[i]), kStreamWarps * 32);
+            ptx::mbar_init(ptx::smem_u32(&sh.xchg[i]), kStreamWarps);
+            ptx::mbar_init(ptx::smem_u32(&sh.zbar[i]), kStreamWarps);
             ptx::mbar_init(ptx::smem_u32(&sh.v_ready[i]), kConvWarps);
             ptx::mbar_init(ptx::smem_u32(&sh.pv_done[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.pv_pair[i]), 1);
         }
-        ptx::mbar_init(ptx::smem_u32(&sh.zbar), kSoftmaxWarps);
         ptx::mbar_init(ptx::smem_u32(&sh.drain_qk), 1);
         ptx::mbar_init(ptx::smem_u32(&sh.drain_pv), 1);
         sh.abort_flag = 0;
@@ -133,14 +148,17 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     const int t0 = split * per_split, t1 = min(n_tiles, t0 + per_split);
     const int n_it = t1 - t0;
     const int n_pairs = (n_it + 1) / 2;   // the softmax warps take two key tiles per step
-    const int64_t out_row0 = (static_cast<int64_t>(b) * prm.Hq + hk * R) * prm.n_splits + split;   // + r * n_splits
+    const int n_parts = kStreams * prm.n_splits;   // partial results per query head in the workspace
+    const int64_t out_row0 = (static_cast<int64_t>(b) * prm.Hq + hk * R) * n_parts + kStreams * split;   // + r * n_parts + stream
 
     if (n_it <= 0) {                      // a split without keys: the merge skips it
-        for (int idx = tid; idx < R * D; idx += kThreads)
-            prm.o_part[(out_row0 + static_cast<int64_t>(idx / D) * prm.n_splits) * D + (idx % D)] = 0.f;
-        if (tid < R) {
-            prm.m_part[out_row0 + static_cast<int64_t>(tid) * prm.n_splits] = -INFINITY;
-            prm.z_part[out_row0 + static_cast<int64_t>(tid) * prm.n_splits] = 0.f;
+        for (int idx = tid; idx < kStreams * R * D; idx += kThreads) {
+            const int g = idx / (R * D), rd = idx % (R * D);
+            prm.o_part[(out_row0 + static_cast<int64_t>(rd / D) * n_parts + g) * D + (rd % D)] = 0.f;
+        }
+        if (tid < kStreams * R) {
+            prm.m_part[out_row0 + static_cast<int64_t>(tid % R) * n_parts + tid / R] = -INFINITY;
+            prm.z_part[out_row0 + static_cast<int64_t>(tid % R) * n_parts + tid / R] = 0.f;
         }
         leave();
         return;
@@ -198,6 +216,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     int last_issued = -1;                 // (producer lane) the last tile whose copies were started
     if (warp == kProducerWarp) {
         // ============================================================ copy producer (one lane)
+        ptx::setmaxnreg_dec<kRegsCtl>();
         if (lane == 0) {
             int head = 0, used = 0, freed = 0;
             // route bits straight from the mask words (the staged tile metadata is not there yet when this loop
@@ -246,14 +265,20 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         const __half2 off = __floats2half2_rn(1152.f, 1152.f);
         constexpr int kPer = T * D / 16 / kConvThreads;   // 16-byte pieces per thread and tile
         const int8_t* v8 = prm.v8 + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.max_len * D;
+        // Piece idx of a tile = 16 bytes (columns 16q .. 16q+15) of one key.  Eight consecutive pieces are the
+        // four pieces of one 64-column half of two adjacent keys: as FP16 they are the even 16-byte chunks of
+        // one key's 128-byte row and the odd ones of the other's (the swizzle flips the parity with the row), so
+        // a quarter warp's 128-bit stores fall into eight different bank groups.
+        auto piece_row = [](int idx) { return ((idx >> 4) << 1) | ((idx >> 2) & 1); };
+        auto piece_q = [](int idx) { return (((idx >> 3) & 1) << 2) | (idx & 3); };
         auto vload = [&](int it, uint4 (&dst)[kPer]) {
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
                 const int idx = cid + kConvThreads * j;
-                const int64_t row = static_cast<int64_t>(t0 + it) * T + (idx >> 3);
+                const int64_t row = static_cast<int64_t>(t0 + it) * T + piece_row(idx);
                 dst[j] = make_uint4(0u, 0u, 0u, 0u);
                 if (it < n_it && row < len) {     // rows past the cache are not read (their P is zero)
-                    const int8_t* src = v8 + row * D + (idx & 7) * 16;
+                    const int8_t* src = v8 + row * D + piece_q(idx) * 16;
                     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                                  : "=r"(dst[j].x), "=r"(dst[j].y), "=r"(dst[j].z), "=r"(dst[j].w)
                                  : "l"(src));
@@ -310,6 +335,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
 
         if (warp == kQkWarp) {
         // ============================================================ QK^T issuer (whole warp, elected-lane issue)
+        ptx::setmaxnreg_dec<kRegsCtl>();
         constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, T, 16);
         constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, T, 16);
         const uint32_t q8_lo = ptx::desc_lo(sbase + kOffQ8, 16);
@@ -352,6 +378,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         wait(&sh.drain_qk, 0, kWDrain);
         } else if (warp == kPvWarp) {
         // ============================================================ PV issuer (whole warp, elected-lane issue)
+        ptx::setmaxnreg_dec<kRegsCtl>();
         constexpr uint32_t kIdescPV = ptx::instr_desc(1, 0, 0, 1, kPRows, D);
         bool ok = true;
         for (int j = 0; j < n_pairs && ok; ++j) {
@@ -366,18 +393,21 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                 const uint32_t b_base = ptx::desc_lo(sbase + kOffV16 + h * kVBytes, kVBytes / 2);
 #pragma unroll
                 for (int k = 0; k < T / 16; ++k)  // 16 keys per step: 32 bytes of a P row, 16 rows (2048 bytes) of V16
-                    ptx::mma_f16_ss_rt(tmem_base + kColO, a_base + (k >> 2) * (1024 >> 4) + 2 * (k & 3), kHi,
-                                       b_base + k * 128, kHi, kIdescPV, (it > 0 || k > 0) ? 1u : 0u);
+                    ptx::mma_f16_ss_rt(tmem_base + kColO + pb * 128, a_base + (k >> 2) * (1024 >> 4) + 2 * (k & 3), kHi,
+                                       b_base + k * 128, kHi, kIdescPV, (j >= kStreams || h > 0 || k > 0) ? 1u : 0u);
                 ptx::mma_commit(ptx::smem_u32(&sh.pv_done[h]));
             }
             if (ok) ptx::mma_commit(ptx::smem_u32(&sh.pv_pair[pb]));
         }
         ptx::mma_commit(ptx::smem_u32(&sh.drain_pv));
         wait(&sh.drain_pv, 0, kWDrain);
+        } else if (warp > kPvWarp) {
+            ptx::setmaxnreg_dec<kRegsCtl>();      // the idle warp of the last group
         } else if (warp >= kConvWarp0) {
         // ============================================================ V8 -> FP16 (sixteen warps, one key tile at a time)
         // V8 never touches shared memory: a thread loads its 16-byte pieces of the next kVDepth tiles straight
         // from the cache into registers (that is the prefetch), converts the oldest and stores FP16.
+        ptx::setmaxnreg_inc<Regs<R>::kConv>();
         bool ok = true;
         for (int it0 = 0; it0 < n_it && ok; it0 += kVDepth) {
 #pragma unroll
@@ -388,7 +418,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                 uint8_t* dst = sm + kOffV16 + bf * kVBytes;
 #pragma unroll
                 for (int j = 0; j < kPer; ++j) {
-                    const int idx = cid + kConvThreads * j, row = idx >> 3, q = idx & 7;   // columns 16q .. 16q+15 of a key
+                    const int idx = cid + kConvThreads * j, row = piece_row(idx), q = piece_q(idx);
                     const uint32_t w[4] = {buf[x][j].x, buf[x][j].y, buf[x][j].z, buf[x][j].w};
                     uint32_t h[8];
 #pragma unroll
@@ -401,14 +431,14 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                         h[2 * y] = *reinterpret_cast<const uint32_t*>(&v0);
                         h[2 * y + 1] = *reinterpret_cast<const uint32_t*>(&v1);
                     }
-                    // slab q / 4, 16-byte chunks 2(q % 4) and + 1 of the key's 128-byte row, swizzled by the row; the
-                    // upper half of the lanes stores its chunks in the other order (no bank conflicts)
+                    // slab q / 4, 16-byte chunks 2(q % 4) and + 1 of the key's 128-byte row, swizzled by the row
                     uint8_t* rowp = dst + (q >> 2) * (kVBytes / 2) + row * 128;
                     const int c0 = 2 * (q & 3), sw = row & 7;
                     uint4* p0 = reinterpret_cast<uint4*>(rowp + ((c0 ^ sw) << 4));
                     uint4* p1 = reinterpret_cast<uint4*>(rowp + (((c0 + 1) ^ sw) << 4));
                     const uint4 a = make_uint4(h[0], h[1], h[2], h[3]), c = make_uint4(h[4], h[5], h[6], h[7]);
-                    if (q < 4) { *p0 = a; *p1 = c; } else { *p1 = c; *p0 = a; }
+                    *p0 = a;
+                    *p1 = c;
                 }
                 vload(it + kVDepth, buf[x]);      // refill: the tile kVDepth ahead
                 ptx::fence_proxy_async_smem();
@@ -417,8 +447,10 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             }
         }
         } else {
-        // ============================================================ softmax (thread = one key of each tile of a pair)
-        const int key = tid;
+        // ============================================================ softmax (thread = one key of each tile of a step)
+        if constexpr (Regs<R>::kSoft < kLaunchRegs) ptx::setmaxnreg_dec<Regs<R>::kSoft>();
+        const int g = warp >> 2, wq = warp & 3;       // stream, TMEM lane quarter
+        const int key = wq * 32 + lane;
         float m_run[R], z_part[R], a_q[R];
         uint32_t p_off[R];
 #pragma unroll
@@ -428,9 +460,17 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             a_q[r] = prm.scale_log2 * sh.dq[r];
             p_off[r] = (key >> 6) * 1024 + r * 128 + ((((key & 63) >> 3) ^ r) << 4) + (key & 7) * 2;
         }
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-        for (int j = 0; j < n_pairs; ++j) {
-            const int pb = j & 1;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(wq * 32) << 16);
+        const uint32_t col_o = kColO + g * 128;
+        const int64_t orow = out_row0 + static_cast<int64_t>(lane < R ? lane : 0) * n_parts + g;   // (lanes < R of quarter 0)
+        if (g >= n_pairs) {
+            // a stream without a step: an empty partial result, which the merge skips
+            for (int idx = key; idx < R * D; idx += kStreamWarps * 32)
+                prm.o_part[(out_row0 + static_cast<int64_t>(idx / D) * n_parts + g) * D + (idx % D)] = 0.f;
+            if (wq == 0 && lane < R) { prm.m_part[orow] = -INFINITY; prm.z_part[orow] = 0.f; }
+        }
+        for (int j = g; j < n_pairs; j += kStreams) {
+            const uint32_t par = (j >> 1) & 1;        // phase parity of this stream's barriers at this step
             const bool two = 2 * j + 1 < n_it;
             bool int8[2];
             float dkt[2], dvt[2];
@@ -444,17 +484,17 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                     int8[h] = route_of(tile); dkt[h] = int8[h] ? dk[tile] : 0.f; dvt[h] = dv[tile];
                 }
             }
-            if (!wait(&sh.s_ready[pb], (j >> 1) & 1, kWS)) break;
+            if (!wait(&sh.s_ready[g], par, kWS)) break;
             ptx::tc_fence_after_sync();
             uint32_t raw[2][RC];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                if constexpr (RC == 4) ptx::tmem_ld32x32_x4(t_lane + (2 * pb + h) * 16, raw[h]);
-                else ptx::tmem_ld32x32_x8(t_lane + (2 * pb + h) * 16, raw[h]);
+                if constexpr (RC == 4) ptx::tmem_ld32x32_x4(t_lane + (2 * g + h) * 16, raw[h]);
+                else ptx::tmem_ld32x32_x8(t_lane + (2 * g + h) * 16, raw[h]);
             }
             ptx::tmem_wait_ld_dep(raw[0], raw[1]);    // ties the registers to the wait: no use of them moves above it
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(ptx::smem_u32(&sh.s_free[pb]));
+            ptx::mbar_arrive(ptx::smem_u32(&sh.s_free[g]));
             float sc[2][R];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -468,28 +508,31 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                 }
             }
             // maximum of the step per row: over the warp (order-preserving integer image of the float), then
-            // over the four warps through shared memory
+            // over the four warps of the stream through shared memory
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 int o = __float_as_int(fmaxf(sc[0][r], sc[1][r]));
                 o = o >= 0 ? o : o ^ 0x7fffffff;
                 o = __reduce_max_sync(0xffffffffu, o);
                 o = o >= 0 ? o : o ^ 0x7fffffff;
-                if (lane == 0) sh.warp_max[pb][warp][r] = __int_as_float(o);
+                if (lane == 0) sh.warp_max[g][wq][r] = __int_as_float(o);
             }
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.xchg[pb]));
-            if (!wait(&sh.xchg[pb], (j >> 1) & 1, kWXchg)) break;
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.xchg[g]));
+            if (!wait(&sh.xchg[g], par, kWXchg)) break;
             bool move = false;
             float mt[R];
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                mt[r] = fmaxf(fmaxf(sh.warp_max[pb][0][r], sh.warp_max[pb][1][r]),
-                              fmaxf(sh.warp_max[pb][2][r], sh.warp_max[pb][3][r]));
-                move |= mt[r] > m_run[r] + kMoveAbove;      // always on the first step (m = -inf)
+                mt[r] = fmaxf(fmaxf(sh.warp_max[g][0][r], sh.warp_max[g][1][r]),
+                              fmaxf(sh.warp_max[g][2][r], sh.warp_max[g][3][r]));
+                move |= mt[r] > m_run[r] + kMoveAbove;      // always on the stream's first step (m = -inf)
             }
-            const int last_it = min(2 * j + 1, n_it - 1);   // the last tile of this step
-            if (move) {                                      // CTA-uniform
+            // The PVs of this stream's previous step have retired: they read the P tiles written below and they
+            // accumulate into the O that a move of m rescales.  (A barrier per stream whose next phase cannot
+            // complete before this step hands P over, so the wait cannot be lapped.)
+            if (j >= kStreams && !wait(&sh.pv_pair[g], par ^ 1u, kWPV)) break;
+            if (move) {                                      // uniform over the stream
                 float alpha_lane = 1.f;
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
@@ -499,60 +542,55 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                     m_run[r] = mn;
                     if (lane == r) alpha_lane = alpha;
                 }
-                if (j > 0 && warp == 0) {
-                    // rows 0..R-1 of O (lanes 0..R-1 of tensor memory) are rescaled once every PV issued so far has
-                    // retired (the last ones are those of step j - 1); the PVs of this step cannot start before this
-                    // warp hands P over
-                    if (!wait(&sh.pv_pair[pb ^ 1], ((j - 1) >> 1) & 1, kWPV)) break;
+                if (j >= kStreams && wq == 0) {
+                    // rows 0..R-1 of this stream's O (lanes 0..R-1 of tensor memory); the PVs of this step cannot
+                    // start before this warp hands P over
                     ptx::tc_fence_after_sync();
 #pragma unroll 1
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[32];
-                        ptx::tmem_ld32(tmem_base + kColO + 32 * c, o);
+                        ptx::tmem_ld32(tmem_base + col_o + 32 * c, o);
                         ptx::tmem_wait_ld_dep(o);
 #pragma unroll
                         for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * alpha_lane);
-                        ptx::tmem_st32(tmem_base + kColO + 32 * c, o);
+                        ptx::tmem_st32(tmem_base + col_o + 32 * c, o);
                     }
                     ptx::tmem_wait_st();
                     ptx::tc_fence_before_sync();
                 }
             }
-            // the PVs that read this pair of P tiles two steps ago have retired (a barrier per pair buffer: its
-            // next phase cannot complete before this step hands P over, so the wait cannot be lapped)
-            if (j >= 2 && !wait(&sh.pv_pair[pb], ((j >> 1) - 1) & 1, kWPV)) break;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                uint8_t* pbuf = sm + kOffP + (2 * pb + h) * kPTile;
+                uint8_t* pbuf = sm + kOffP + (2 * g + h) * kPTile;
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    const float p = exp2f(sc[h][r] - m_run[r]);
+                    float p;
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(sc[h][r] - m_run[r]));
                     z_part[r] += p;
                     *reinterpret_cast<__half*>(pbuf + p_off[r]) = __float2half_rn(p * dvt[h]);
                 }
             }
             ptx::fence_proxy_async_smem();
-            ptx::mbar_arrive(ptx::smem_u32(&sh.p_ready[pb]));
-            if (j == n_pairs - 1) {
-                // ---- (m, z, O~) of this split to the workspace
+            ptx::mbar_arrive(ptx::smem_u32(&sh.p_ready[g]));
+            if (j + kStreams >= n_pairs) {
+                // ---- the stream's last step: (m, z, O~) to the workspace
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     float z = z_part[r];
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-                    if (lane == 0) sh.zsum[warp][r] = z;
+                    if (lane == 0) sh.zsum[g][wq][r] = z;
                 }
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.zbar));
-                if (warp != 0) break;
-                if (!wait(&sh.zbar, 0, kWXchg)) break;
-                if (!wait(&sh.pv_done[last_it & 1], (last_it >> 1) & 1, kWPV)) break;
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.zbar[g]));
+                if (wq != 0) break;
+                if (!wait(&sh.zbar[g], 0, kWXchg)) break;
+                if (!wait(&sh.pv_pair[g], par, kWPV)) break;      // the PVs of this step
                 ptx::tc_fence_after_sync();
-                const int64_t orow = out_row0 + static_cast<int64_t>(lane < R ? lane : 0) * prm.n_splits;
 #pragma unroll 1
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
-                    ptx::tmem_ld32(tmem_base + kColO + 32 * c, o);
+                    ptx::tmem_ld32(tmem_base + col_o + 32 * c, o);
                     ptx::tmem_wait_ld_dep(o);
                     if (lane < R) {
                         float4* dstp = reinterpret_cast<float4*>(prm.o_part + orow * D + 32 * c);
@@ -567,7 +605,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
 #pragma unroll
                     for (int r = 0; r < R; ++r) if (lane == r) mine = m_run[r];
                     prm.m_part[orow] = mine;
-                    prm.z_part[orow] = sh.zsum[0][lane] + sh.zsum[1][lane] + sh.zsum[2][lane] + sh.zsum[3][lane];
+                    prm.z_part[orow] = sh.zsum[g][0][lane] + sh.zsum[g][1][lane] + sh.zsum[g][2][lane] + sh.zsum[g][3][lane];
                 }
                 ptx::tc_fence_before_sync();
             }
@@ -616,6 +654,12 @@ int launch_r(const DecodeParams& prm, const CUtensorMap& tk8, const CUtensorMap&
     auto kernel = prm.k16 != nullptr ? decode_umma_kernel<R, true> : decode_umma_kernel<R, false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return static_cast<int>(e);
+    // the register split inside the kernel adds up to kThreads * kLaunchRegs: never launch a build that was
+    // given fewer (its setmaxnreg.inc would wait for registers that do not exist)
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, kernel);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    if (fa.numRegs < kLaunchRegs) return TILEMIX_ERR_UNSUPPORTED;
     const dim3 grid(prm.n_splits, prm.Hk, prm.B);
     // programmatic dependent launch: this grid's set-up overlaps the tail of the prepare kernel
     cudaLaunchConfig_t cfg = {};
