@@ -32,10 +32,9 @@ namespace {
 
 constexpr int D = 128, T = 128;
 constexpr int kUnit = T * D;              // bytes of a ring unit
-constexpr int kUnits = 9;
-constexpr int kSlots = 16;                // barrier slots of key tiles in the ring (at most kUnits fit)
-constexpr int kVDepth = 6;                // V8 tiles a conversion thread keeps in flight in its registers
-constexpr int kVBytes = T * D * 2;        // FP16 copy of a V tile: two 64-column slabs of 16 KB
+constexpr int kUnits = 11;
+constexpr int kSlots = 8;                 // barrier slots of tiles in the ring (at most kUnits / 2 tiles fit)
+constexpr int kVHalf = (T / 2) * D * 2;   // FP16 copy of half a V tile (64 keys): two 64-column slabs of 8 KB
 constexpr int kPRows = 64;                // M of the PV product
 constexpr int kPTile = 2048;              // P of a key tile: rows 0..7 of two 64-key slabs (1 KB each)
 constexpr int kMetaTiles = 256;
@@ -48,7 +47,7 @@ constexpr int kOffQ8 = kOffP + 4 * kPTile;       // 8 rows x 128 bytes
 constexpr int kOffQ16 = kOffQ8 + 1024;           // two slabs of 8 rows x 128 bytes
 constexpr int kOffRing = kOffQ16 + 2048 + 1024;
 constexpr int kOffV16 = kOffRing + kUnits * kUnit;
-constexpr int kOffMeta = kOffV16 + 2 * kVBytes;
+constexpr int kOffMeta = kOffV16 + 2 * kVHalf;
 constexpr int kOffSmall = kOffMeta + kMetaTiles * 8;
 static_assert(kOffRing % 1024 == 0 && kOffV16 % 1024 == 0, "swizzled tiles start on 1 KB boundaries");
 
@@ -59,30 +58,19 @@ static_assert(kOffRing % 1024 == 0 && kOffV16 % 1024 == 0, "swizzled tiles start
 constexpr int kStreams = 2, kStreamWarps = 4, kSoftmaxWarps = kStreams * kStreamWarps, kConvWarps = 16;
 constexpr int kConvWarp0 = kSoftmaxWarps, kProducerWarp = kConvWarp0 + kConvWarps;
 constexpr int kQkWarp = kProducerWarp + 1, kPvWarp = kQkWarp + 1;
-constexpr int kThreads = (kPvWarp + 2) * 32;   // one idle warp completes the last group of four (setmaxnreg)
+constexpr int kThreads = (kPvWarp + 1) * 32;
 constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kTmemCols = 512;            // S^T: four buffers of 16 columns from column 0; O of stream g: 128 + 128 g
 constexpr uint32_t kColO = 128;
-// Registers: the block is launched with kLaunchRegs per thread; the conversion warps, which hold kVDepth tiles of V8
-// in flight, take more, the others hand theirs back.  The split must add up to the launch allotment exactly
-// (setmaxnreg.inc waits for registers that other warps release: a split above the allotment would wait for ever;
-// the host refuses to launch when the compiler planned for fewer registers than kLaunchRegs).
-constexpr int kLaunchRegs = 72, kRegsCtl = 40;
-template <int R> struct Regs {
-    static constexpr int kConv = R == 8 ? 80 : 88, kSoft = R == 8 ? 72 : 56;
-    static_assert(kConvThreads * kConv + kSoftmaxWarps * 32 * kSoft + 4 * 32 * kRegsCtl == kThreads * kLaunchRegs,
-                  "setmaxnreg split");
-};
-static_assert(kThreads == 896 && kThreads % 128 == 0, "warp groups of four");
 constexpr float kMoveAbove = 8.f;         // m moves when a step's maximum exceeds it by more than 2^8
 
 struct Small {
     uint64_t full[kSlots], freeb[kSlots];
     uint64_t s_ready[2], s_free[2], p_ready[2], xchg[2];      // per pair buffer
-    uint64_t v_ready[2], pv_done[2];                          // per V16 buffer (tile parity)
+    uint64_t v_ready[2], pv_done[2];                          // per V16 buffer (half of a tile)
     uint64_t pv_pair[2];                                      // per pair buffer: the PVs of a step have retired
     uint64_t zbar[kStreams], drain_qk, drain_pv;
-    uint32_t slot_info[kSlots];           // ring units of the key tile in a slot: byte 0, second FP16 slab: byte 1
+    uint32_t slot_info[kSlots];           // ring units of the tile in a slot: K (byte 0), second K slab (1), V (2)
     float warp_max[kStreams][kStreamWarps][8];
     float zsum[kStreams][kStreamWarps][8];
     float dq[8];
@@ -112,7 +100,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
             ptx::mbar_init(ptx::smem_u32(&sh.full[s]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh.freeb[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh.freeb[s]), 1 + kConvWarps);
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh.s_ready[i]), 1);
@@ -120,7 +108,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             ptx::mbar_init(ptx::smem_u32(&sh.p_ready[i]), kStreamWarps * 32);
             ptx::mbar_init(ptx::smem_u32(&sh.xchg[i]), kStreamWarps);
             ptx::mbar_init(ptx::smem_u32(&sh.zbar[i]), kStreamWarps);
-            ptx::mbar_init(ptx::smem_u32(&sh.v_ready[i]), kConvWarps);
+            ptx::mbar_init(ptx::smem_u32(&sh.v_ready[i]), kConvWarps / 2);
             ptx::mbar_init(ptx::smem_u32(&sh.pv_done[i]), 1);
             ptx::mbar_init(ptx::smem_u32(&sh.pv_pair[i]), 1);
         }
@@ -216,80 +204,57 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     int last_issued = -1;                 // (producer lane) the last tile whose copies were started
     if (warp == kProducerWarp) {
         // ============================================================ copy producer (one lane)
-        ptx::setmaxnreg_dec<kRegsCtl>();
         if (lane == 0) {
+            const int8_t* v8g = prm.v8 + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.max_len * D;
             int head = 0, used = 0, freed = 0;
-            // route bits straight from the mask words (the staged tile metadata is not there yet when this loop
-            // starts), one word kept in a register
-            uint32_t cw_idx = 0xffffffffu, cw = 0u;
-            auto route_cached = [&](int tile) -> bool {
-                if (wrow == nullptr) return false;
-                const uint32_t grp = static_cast<uint32_t>(tile / prm.G);
-                if ((grp >> 5) != cw_idx) { cw_idx = grp >> 5; cw = wrow[cw_idx]; }
-                return (cw >> (grp & 31u)) & 1u;
-            };
+            // Route bits straight from the mask words (the staged tile metadata is not there yet when this loop
+            // starts), without a division per tile: group index and position inside the group advance with the
+            // tile, one mask word is kept in a register, and the routes of the tiles in the ring are remembered
+            // as bits (tile it -> bit it % 32) for the moment their units come back.
+            uint32_t grp = static_cast<uint32_t>(t0 / prm.G), in_grp = static_cast<uint32_t>(t0 % prm.G);
+            uint32_t cw = wrow != nullptr ? wrow[grp >> 5] : 0u, routes = 0u;
             for (int it = 0; it < n_it; ++it) {
-                const bool i8 = route_cached(t0 + it);
-                const int need = i8 ? 1 : 2;
+                const bool i8 = (cw >> (grp & 31u)) & 1u;
+                routes = (routes & ~(1u << (it & 31))) | (static_cast<uint32_t>(i8) << (it & 31));
+                if (++in_grp == static_cast<uint32_t>(prm.G)) {
+                    in_grp = 0;
+                    ++grp;
+                    if ((grp & 31u) == 0u && wrow != nullptr && it + 1 < n_it) cw = wrow[grp >> 5];
+                }
+                const int need = i8 ? 2 : 3;
                 bool ok = true;
                 while (used + need > kUnits || it - freed >= kSlots) {
                     if (!wait(&sh.freeb[freed % kSlots], (freed / kSlots) & 1, kWFree)) { ok = false; break; }
-                    used -= route_cached(t0 + freed) ? 1 : 2;
+                    used -= ((routes >> (freed & 31)) & 1u) ? 2 : 3;
                     ++freed;
                 }
                 if (!ok) break;
                 const int s = it % kSlots;
-                const uint32_t u0 = head, u1 = (head + 1) % kUnits;
+                const uint32_t u0 = head, u1 = (head + 1) % kUnits, u2 = (head + 2) % kUnits;
+                const uint32_t uv = i8 ? u1 : u2;
                 head = (head + need) % kUnits;
                 used += need;
-                *reinterpret_cast<volatile uint32_t*>(&sh.slot_info[s]) = u0 | (u1 << 8);
+                *reinterpret_cast<volatile uint32_t*>(&sh.slot_info[s]) = u0 | (u1 << 8) | (uv << 16);
                 if (it == prm.test_drop_tile) continue;   // testing aid: this tile never lands, the consumers' waits run out
                 const int tile = t0 + it;
+                const uint32_t rows = static_cast<uint32_t>(min(T, len - tile * T));
                 const uint32_t bar = ptx::smem_u32(&sh.full[s]);
                 // the tiled copies always bring a whole box (rows past the cache are stale or zero-filled and are
-                // masked as keys)
-                ptx::mbar_arrive_expect_tx(bar, i8 ? kUnit : 2 * kUnit);
+                // masked as keys); the plain copy of V8 brings the rows that exist
+                ptx::mbar_arrive_expect_tx(bar, (i8 ? kUnit : 2 * kUnit) + rows * D);
                 if (i8) {
                     ptx::tma_load_4d(sbase + kOffRing + u0 * kUnit, &tm_k8, bar, 0, tile * T, hk, b);
                 } else {
                     ptx::tma_load_4d(sbase + kOffRing + u0 * kUnit, &tm_k16, bar, 0, tile * T, hk, b);
                     ptx::tma_load_4d(sbase + kOffRing + u1 * kUnit, &tm_k16, bar, 64, tile * T, hk, b);
                 }
+                ptx::bulk_load_1d(sbase + kOffRing + uv * kUnit, v8g + static_cast<int64_t>(tile) * T * D, rows * D, bar);
                 last_issued = it;
             }
         }
     } else {
-        // ---- everyone but the producer: the first V8 loads go out, then the operand tiles of Q are made ----------
+        // ---- everyone but the producer: the operand tiles of Q are made while the first copies fly -----------------
         const int nid = tid < kProducerWarp * 32 ? tid : tid - 32;
-        const int cid = tid - kConvWarp0 * 32;
-        const __half2 off = __floats2half2_rn(1152.f, 1152.f);
-        constexpr int kPer = T * D / 16 / kConvThreads;   // 16-byte pieces per thread and tile
-        const int8_t* v8 = prm.v8 + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.max_len * D;
-        // Piece idx of a tile = 16 bytes (columns 16q .. 16q+15) of one key.  Eight consecutive pieces are the
-        // four pieces of one 64-column half of two adjacent keys: as FP16 they are the even 16-byte chunks of
-        // one key's 128-byte row and the odd ones of the other's (the swizzle flips the parity with the row), so
-        // a quarter warp's 128-bit stores fall into eight different bank groups.
-        auto piece_row = [](int idx) { return ((idx >> 4) << 1) | ((idx >> 2) & 1); };
-        auto piece_q = [](int idx) { return (((idx >> 3) & 1) << 2) | (idx & 3); };
-        auto vload = [&](int it, uint4 (&dst)[kPer]) {
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const int idx = cid + kConvThreads * j;
-                const int64_t row = static_cast<int64_t>(t0 + it) * T + piece_row(idx);
-                dst[j] = make_uint4(0u, 0u, 0u, 0u);
-                if (it < n_it && row < len) {     // rows past the cache are not read (their P is zero)
-                    const int8_t* src = v8 + row * D + piece_q(idx) * 16;
-                    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(dst[j].x), "=r"(dst[j].y), "=r"(dst[j].z), "=r"(dst[j].w)
-                                 : "l"(src));
-                }
-            }
-        };
-        uint4 buf[kVDepth][kPer];
-        if (warp >= kConvWarp0 && warp < kProducerWarp) {
-#pragma unroll
-            for (int x = 0; x < kVDepth; ++x) vload(x, buf[x]);
-        }
         {
             // rows R..7 of the P and Q tiles are never written: zero them once (finite values in the unused rows)
             uint4* z = reinterpret_cast<uint4*>(sm + kOffP);
@@ -335,7 +300,6 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
 
         if (warp == kQkWarp) {
         // ============================================================ QK^T issuer (whole warp, elected-lane issue)
-        ptx::setmaxnreg_dec<kRegsCtl>();
         constexpr uint32_t kIdescQK8 = ptx::instr_desc(2, 1, 0, 0, T, 16);
         constexpr uint32_t kIdescQK16 = ptx::instr_desc(1, 0, 0, 0, T, 16);
         const uint32_t q8_lo = ptx::desc_lo(sbase + kOffQ8, 16);
@@ -378,7 +342,6 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         wait(&sh.drain_qk, 0, kWDrain);
         } else if (warp == kPvWarp) {
         // ============================================================ PV issuer (whole warp, elected-lane issue)
-        ptx::setmaxnreg_dec<kRegsCtl>();
         constexpr uint32_t kIdescPV = ptx::instr_desc(1, 0, 0, 1, kPRows, D);
         bool ok = true;
         for (int j = 0; j < n_pairs && ok; ++j) {
@@ -387,68 +350,83 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             for (int h = 0; h < 2; ++h) {
                 const int it = 2 * j + h;
                 if (it >= n_it) break;
-                if (!wait(&sh.v_ready[h], j & 1, kWV)) { ok = false; break; }
-                ptx::tc_fence_after_sync();
                 const uint32_t a_base = ptx::desc_lo(sbase + kOffP + (2 * pb + h) * kPTile, 16);
-                const uint32_t b_base = ptx::desc_lo(sbase + kOffV16 + h * kVBytes, kVBytes / 2);
+                // the FP16 copy of V arrives in two halves of 64 keys, each in its own buffer
 #pragma unroll
-                for (int k = 0; k < T / 16; ++k)  // 16 keys per step: 32 bytes of a P row, 16 rows (2048 bytes) of V16
-                    ptx::mma_f16_ss_rt(tmem_base + kColO + pb * 128, a_base + (k >> 2) * (1024 >> 4) + 2 * (k & 3), kHi,
-                                       b_base + k * 128, kHi, kIdescPV, (j >= kStreams || h > 0 || k > 0) ? 1u : 0u);
-                ptx::mma_commit(ptx::smem_u32(&sh.pv_done[h]));
+                for (int hf = 0; hf < 2; ++hf) {
+                    if (!wait(&sh.v_ready[hf], it & 1, kWV)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t b_base = ptx::desc_lo(sbase + kOffV16 + hf * kVHalf, kVHalf / 2);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)   // 16 keys per step: 32 bytes of a P row, 16 rows (2048 bytes) of V16
+                        ptx::mma_f16_ss_rt(tmem_base + kColO + pb * 128, a_base + hf * (1024 >> 4) + 2 * k, kHi,
+                                           b_base + k * 128, kHi, kIdescPV, (j >= kStreams || h > 0 || hf > 0 || k > 0) ? 1u : 0u);
+                    ptx::mma_commit(ptx::smem_u32(&sh.pv_done[hf]));
+                }
+                if (!ok) break;
             }
             if (ok) ptx::mma_commit(ptx::smem_u32(&sh.pv_pair[pb]));
         }
         ptx::mma_commit(ptx::smem_u32(&sh.drain_pv));
         wait(&sh.drain_pv, 0, kWDrain);
-        } else if (warp > kPvWarp) {
-            ptx::setmaxnreg_dec<kRegsCtl>();      // the idle warp of the last group
         } else if (warp >= kConvWarp0) {
-        // ============================================================ V8 -> FP16 (sixteen warps, one key tile at a time)
-        // V8 never touches shared memory: a thread loads its 16-byte pieces of the next kVDepth tiles straight
-        // from the cache into registers (that is the prefetch), converts the oldest and stores FP16.
-        ptx::setmaxnreg_inc<Regs<R>::kConv>();
-        bool ok = true;
-        for (int it0 = 0; it0 < n_it && ok; it0 += kVDepth) {
+        // ============================================================ V8 -> FP16 (two groups of eight warps)
+        // Group hf converts keys 64 hf .. 64 hf + 63 of every tile into its own FP16 buffer (a role's step is mostly
+        // the fixed cost of its waits and its proxy fence: two groups in parallel halve it per tile).  A thread takes
+        // its two 16-byte pieces of a landed V8 tile into registers (the ring unit goes back to the producer at
+        // once) and converts them when the PV that read the buffer last has retired.
+        // Piece idx of a half = columns 16q .. 16q+15 of one of its 64 keys.  Eight consecutive pieces are the four
+        // pieces of one 64-column half of two adjacent keys: as FP16 they are the even 16-byte chunks of one key's
+        // 128-byte row and the odd ones of the other's (the swizzle flips the parity with the row), so a quarter
+        // warp's 128-bit stores fall into eight different bank groups.
+        const int hf = (warp - kConvWarp0) >> 3;
+        const int cid = ((warp - kConvWarp0) & 7) * 32 + lane;
+        constexpr int kGroupThreads = kConvThreads / 2, kPer = (T / 2) * D / 16 / kGroupThreads;
+        const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+        uint8_t* vbuf = sm + kOffV16 + hf * kVHalf;
+        for (int it = 0; it < n_it; ++it) {
+            const int s = it % kSlots;
+            if (!wait(&sh.full[s], (it / kSlots) & 1, kWFull)) break;
+            const uint32_t info = *reinterpret_cast<volatile uint32_t*>(&sh.slot_info[s]);
+            const uint8_t* src = sm + kOffRing + ((info >> 16) & 0xffu) * kUnit + hf * (T / 2) * D;
+            uint4 in[kPer];
 #pragma unroll
-            for (int x = 0; x < kVDepth; ++x) {
-                const int it = it0 + x, bf = it & 1;
-                if (it >= n_it) break;
-                if (it >= 2 && !wait(&sh.pv_done[bf], ((it >> 1) - 1) & 1, kWPV)) { ok = false; break; }   // the PV that read this V16 buffer
-                uint8_t* dst = sm + kOffV16 + bf * kVBytes;
-#pragma unroll
-                for (int j = 0; j < kPer; ++j) {
-                    const int idx = cid + kConvThreads * j, row = piece_row(idx), q = piece_q(idx);
-                    const uint32_t w[4] = {buf[x][j].x, buf[x][j].y, buf[x][j].z, buf[x][j].w};
-                    uint32_t h[8];
-#pragma unroll
-                    for (int y = 0; y < 4; ++y) {
-                        // half2(1024 + (x + 128)) - 1152 = half2(x), exactly
-                        const uint32_t u = w[y] ^ 0x80808080u;
-                        uint32_t lo = __byte_perm(u, 0x64646464u, 0x4140), hi = __byte_perm(u, 0x64646464u, 0x4342);
-                        const __half2 v0 = __hsub2(*reinterpret_cast<const __half2*>(&lo), off);
-                        const __half2 v1 = __hsub2(*reinterpret_cast<const __half2*>(&hi), off);
-                        h[2 * y] = *reinterpret_cast<const uint32_t*>(&v0);
-                        h[2 * y + 1] = *reinterpret_cast<const uint32_t*>(&v1);
-                    }
-                    // slab q / 4, 16-byte chunks 2(q % 4) and + 1 of the key's 128-byte row, swizzled by the row
-                    uint8_t* rowp = dst + (q >> 2) * (kVBytes / 2) + row * 128;
-                    const int c0 = 2 * (q & 3), sw = row & 7;
-                    uint4* p0 = reinterpret_cast<uint4*>(rowp + ((c0 ^ sw) << 4));
-                    uint4* p1 = reinterpret_cast<uint4*>(rowp + (((c0 + 1) ^ sw) << 4));
-                    const uint4 a = make_uint4(h[0], h[1], h[2], h[3]), c = make_uint4(h[4], h[5], h[6], h[7]);
-                    *p0 = a;
-                    *p1 = c;
-                }
-                vload(it + kVDepth, buf[x]);      // refill: the tile kVDepth ahead
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.v_ready[bf]));
+            for (int j = 0; j < kPer; ++j) {
+                const int idx = cid + kGroupThreads * j;
+                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = (((idx >> 3) & 1) << 2) | (idx & 3);
+                in[j] = *reinterpret_cast<const uint4*>(src + row * D + q * 16);
             }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.freeb[s]));    // the V8 tile has been read
+            if (it >= 1 && !wait(&sh.pv_done[hf], (it - 1) & 1, kWPV)) break;   // the PV that read this buffer
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const int idx = cid + kGroupThreads * j;
+                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = (((idx >> 3) & 1) << 2) | (idx & 3);
+                const uint32_t w[4] = {in[j].x, in[j].y, in[j].z, in[j].w};
+                uint32_t h[8];
+#pragma unroll
+                for (int y = 0; y < 4; ++y) {
+                    // half2(1024 + (x + 128)) - 1152 = half2(x), exactly
+                    const uint32_t u = w[y] ^ 0x80808080u;
+                    uint32_t lo = __byte_perm(u, 0x64646464u, 0x4140), hi = __byte_perm(u, 0x64646464u, 0x4342);
+                    const __half2 v0 = __hsub2(*reinterpret_cast<const __half2*>(&lo), off);
+                    const __half2 v1 = __hsub2(*reinterpret_cast<const __half2*>(&hi), off);
+                    h[2 * y] = *reinterpret_cast<const uint32_t*>(&v0);
+                    h[2 * y + 1] = *reinterpret_cast<const uint32_t*>(&v1);
+                }
+                // slab q / 4, 16-byte chunks 2(q % 4) and + 1 of the key's 128-byte row, swizzled by the row
+                uint8_t* rowp = vbuf + (q >> 2) * (kVHalf / 2) + row * 128;
+                const int c0 = 2 * (q & 3), sw = row & 7;
+                *reinterpret_cast<uint4*>(rowp + ((c0 ^ sw) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+                *reinterpret_cast<uint4*>(rowp + (((c0 + 1) ^ sw) << 4)) = make_uint4(h[4], h[5], h[6], h[7]);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh.v_ready[hf]));
         }
         } else {
         // ============================================================ softmax (thread = one key of each tile of a step)
-        if constexpr (Regs<R>::kSoft < kLaunchRegs) ptx::setmaxnreg_dec<Regs<R>::kSoft>();
         const int g = warp >> 2, wq = warp & 3;       // stream, TMEM lane quarter
         const int key = wq * 32 + lane;
         float m_run[R], z_part[R], a_q[R];
@@ -654,12 +632,6 @@ int launch_r(const DecodeParams& prm, const CUtensorMap& tk8, const CUtensorMap&
     auto kernel = prm.k16 != nullptr ? decode_umma_kernel<R, true> : decode_umma_kernel<R, false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return static_cast<int>(e);
-    // the register split inside the kernel adds up to kThreads * kLaunchRegs: never launch a build that was
-    // given fewer (its setmaxnreg.inc would wait for registers that do not exist)
-    cudaFuncAttributes fa;
-    e = cudaFuncGetAttributes(&fa, kernel);
-    if (e != cudaSuccess) return static_cast<int>(e);
-    if (fa.numRegs < kLaunchRegs) return TILEMIX_ERR_UNSUPPORTED;
     const dim3 grid(prm.n_splits, prm.Hk, prm.B);
     // programmatic dependent launch: this grid's set-up overlaps the tail of the prepare kernel
     cudaLaunchConfig_t cfg = {};
