@@ -513,19 +513,30 @@ int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     g->T_mask = static_cast<int>(ceil_div(p->max_len, static_cast<int64_t>(p->group) * p->tile_n));
     g->W = static_cast<int>(ceil_div(g->T_mask, 32));
     int splits = p->n_splits;
+    const bool umma = p->head_dim == 128 && p->tile_n == 128;   // the tcgen05 form of the step (decode_umma.cu)
     if (splits == 0) {
-        // at most two full waves of two CTAs per SM over the whole batch (measured: more splits cost
-        // more in per-CTA set-up and merge than they gain, and a third, partial wave idles a quarter
-        // of the GPU), at least two key tiles per split
-        const int64_t want = (148 * 2 * 2) / (static_cast<int64_t>(p->batch) * p->heads_kv);
-        splits = static_cast<int>(want < 1 ? 1 : want);
-        const int cap = g->n_blk / 2 > 0 ? g->n_blk / 2 : 1;
-        if (splits > cap) splits = cap;
+        if (umma) {
+            // one CTA per SM, HBM-bound once every SM streams: a single wave, as many splits as fit into it
+            // (measured at 8 x 8 KV heads and 32K keys: 2 splits = 128 CTAs 104 us, 9 splits = 3.9 waves 123 us),
+            // at least four key tiles per split
+            const int64_t want = 148 / (static_cast<int64_t>(p->batch) * p->heads_kv);
+            splits = static_cast<int>(want < 1 ? 1 : want);
+            const int cap = g->n_blk / 4 > 0 ? g->n_blk / 4 : 1;
+            if (splits > cap) splits = cap;
+        } else {
+            // at most two full waves of two CTAs per SM over the whole batch (measured: more splits cost
+            // more in per-CTA set-up and merge than they gain, and a third, partial wave idles a quarter
+            // of the GPU), at least two key tiles per split
+            const int64_t want = (148 * 2 * 2) / (static_cast<int64_t>(p->batch) * p->heads_kv);
+            splits = static_cast<int>(want < 1 ? 1 : want);
+            const int cap = g->n_blk / 2 > 0 ? g->n_blk / 2 : 1;
+            if (splits > cap) splits = cap;
+        }
     }
     if (splits > g->n_blk) splits = g->n_blk;
     if (splits > 65535) return TILEMIX_ERR_UNSUPPORTED;
     g->n_splits = splits;
-    g->n_parts = (p->head_dim == 128 && p->tile_n == 128) ? 2 * splits : splits;
+    g->n_parts = umma ? 2 * splits : splits;
     const size_t rows = static_cast<size_t>(p->batch) * p->heads_q * g->n_parts;
     g->o_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
     g->mz_bytes = (rows * sizeof(float) + 255) / 256 * 256;
