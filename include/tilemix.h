@@ -267,9 +267,12 @@ int tilemix_attention_fwd_varlen(const tilemix_problem_t* p, const tilemix_varle
  * scale is folded into the probability before the PV sum (FP32 accumulation), O is written as FP16.
  * Only the K copy a group is routed to is read, so the bytes per cached token are 2*d (INT8 route)
  * or 3*d (FP16 route).  The keys are split over n_splits CTAs per (b, h_k); every CTA serves the
- * H_q/H_k query heads of its KV head (their rows fill a warp-level tensor-core tile); a second
- * kernel merges the partial results.
- * Supported: head_dim 64 or 128, tile_n 64 or 128, H_q/H_k in {1, 2, 4, 8}. */
+ * H_q/H_k query heads of its KV head; a second kernel merges the partial results.
+ * Supported: head_dim 64 or 128, tile_n 64 or 128, H_q/H_k in {1, 2, 4, 8}.  Two forms of the step
+ * kernel: head_dim 128 with tile_n 128 runs on tcgen05 MMAs (keys are the rows of S^T = K Q^T, one CTA
+ * per SM, one wave of CTAs when n_splits is left to the library, two partial results per split); the
+ * other shapes run on warp-level MMAs (the query rows fill a 16-row tile).  Same arithmetic, same
+ * results up to the order of the FP32 sums. */
 typedef struct tilemix_decode {
     int32_t batch, heads_q, heads_kv, head_dim;
     int32_t max_len;       /* token capacity of the caches (their token stride)             */
@@ -296,7 +299,8 @@ size_t tilemix_decode_workspace_size(const tilemix_decode_t* p);
  *   q_i8_out / q_scale_out  nullable INT8 [B, Hq, d] / FP32 [B, Hq]: the quantised query the
  *              kernel used (for checking)
  * Three kernels are enqueued on `stream` (preparation of the lengths and the status record, the step over the
- * splits, the merge).  Errors as for the other entry points; tilemix_read_status on the workspace reports what the
+ * splits, the merge; in the tcgen05 form the last two are programmatic dependent launches, so that their set-up
+ * overlaps the kernel before them).  Errors as for the other entry points; tilemix_read_status on the workspace reports what the
  * kernel itself found (a bounded wait that ran out, or the missing FP16 cache above). */
 int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const void* k_f16,
                           const int8_t* k_i8, const float* k_scale, const int8_t* v_i8,

@@ -585,6 +585,7 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     prm.test_drop_tile = g_test_drop.load() == 2 ? 1 : -1;
     int32_t* len_ws = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + kDecodeStatusBytes);
     prm.cache_len = len_ws;
+    prm.cache_len_raw = cache_len;
     uint8_t* ws = static_cast<uint8_t*>(workspace) + kDecodeStatusBytes + decode_len_bytes(p->batch);
     prm.o_part = reinterpret_cast<float*>(ws);
     prm.m_part = reinterpret_cast<float*>(ws + g.o_bytes);

@@ -19,7 +19,8 @@ struct DecodeParams {
     const int8_t* v8;
     const float* v_scale;
     const uint32_t* words;
-    const int32_t* cache_len;
+    const int32_t* cache_len;       // clamped copy in the workspace (written by the prepare kernel)
+    const int32_t* cache_len_raw;   // the caller's array
     float* o_part;   // [B, Hq, n_splits, D]
     float* m_part;   // [B, Hq, n_splits]
     float* z_part;

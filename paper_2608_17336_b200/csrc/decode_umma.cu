@@ -6,19 +6,22 @@
 //
 //   S^T[128 keys x 16] = K_tile Q^T     A = the key tile as it lands in shared memory (K-major, 128-byte swizzle:
 //                                       INT8 rows of 128 bytes, or two 64-column slabs of FP16 rows), B = the R
-//                                       query rows of this KV head padded to 16 (INT8 copy quantised here, or FP16).
-//                                       Keys are the M rows, so every softmax thread owns one key (one TMEM lane)
-//                                       and R scores; kind::i8 or kind::f16 by the tile's routing bit.
+//                                       query rows of this KV head (INT8 copy quantised here, or FP16).  Keys are the
+//                                       M rows, so every softmax thread owns one key (one TMEM lane) and R scores;
+//                                       kind::i8 or kind::f16 by the tile's routing bit.
 //   P[R x 128 keys]                     2^(s - m) * delta_V rounded to FP16, written by the key's thread into a
-//                                       K-major operand tile (rows >= R stay zero); the row maximum m is shared by
-//                                       the CTA and lazy: it moves only when a tile's maximum exceeds it by 2^8.
-//   V16[128 keys x 128] = FP16(V8)      eight warps convert the INT8 rows exactly (1024 + (x + 128) as FP16 bits,
-//                                       minus 1152) and store them in the MN-major, 128-byte-swizzled layout.
+//                                       K-major operand tile; the row maximum m is shared by a stream's four warps
+//                                       and lazy: it moves only when a step's maximum exceeds it by 2^8.
+//   V16[64 keys x 128] = FP16(V8)       two groups of eight warps convert the INT8 rows exactly (1024 + (x + 128) as
+//                                       FP16 bits, minus 1152), half a tile each, into the MN-major swizzled layout.
 //   O[64 x 128] (+)= P V16              kind::f16, accumulator in tensor memory; rows 0..R-1 are the output.
 //
-// Warps: 0-3 softmax (TMEM lane quarters 0-3), 4-11 conversion, 12 copy producer, 13 MMA issuer.  Operands travel
-// through a ring of 16 KB units (K8 tile, FP16 K slab, V8 tile: one unit each, so an INT8-routed tile takes two and
-// an FP16-routed tile three); S^T, P and V16 are double-buffered.  Every wait is bounded.
+// Warps: 0-7 softmax (two independent streams of four warps, see below), 8-23 conversion, 24 copy producer, 25 QK^T
+// issuer, 26 PV issuer.  K8 / FP16 K slabs / V8 travel through a ring of eleven 16 KB units (an INT8-routed tile
+// takes two, an FP16-routed tile three); what bounds the step is the data in flight -- the loaded HBM latency is
+// several microseconds, so a CTA per SM keeps ~170 KB on the way -- and the fixed cost of each role's waits, which is
+// why every role is either duplicated (softmax streams, conversion groups) or split in two (the issuers).
+// Every wait is bounded; a CTA that gives up records a status, drains what is in flight and returns.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math.h>
@@ -129,8 +132,10 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         __syncthreads();
         if (warp == kProducerWarp) ptx::tmem_dealloc(tmem_base, kTmemCols);
     };
-    ptx::griddep_wait();                  // the prepare kernel's clamped lengths and cleared status record
-    const int len = prm.cache_len[b];     // clamped to [0, max_len] by the prepare kernel
+    // This grid may run beside the prepare kernel (programmatic dependent launch): it takes the length from the
+    // caller's array with the same clamp, and waits for the prepare kernel (which clears the status record) only
+    // where it is about to write that record.
+    const int len = min(max(prm.cache_len_raw[b], 0), prm.max_len);
     const int n_tiles = (len + T - 1) / T;
     const int per_split = (n_tiles + prm.n_splits - 1) / prm.n_splits;
     const int t0 = split * per_split, t1 = min(n_tiles, t0 + per_split);
@@ -167,6 +172,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         int fp16_group = 0;
         for (int tile = t0 + tid; tile < t1; tile += kThreads) fp16_group |= route_of(tile) ? 0 : 1;
         if (__syncthreads_or(fp16_group)) {
+            ptx::griddep_wait();
             if (tid == 0 && atomicCAS(&prm.status[0], 0, TILEMIX_ERR_NULL) == 0) {
                 prm.status[1] = 16; prm.status[2] = t0; prm.status[3] = 1;
             }
@@ -189,6 +195,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
                 if (*abort_flag) return false;
                 if (ptx::globaltimer_ns() - start > prm.wait_limit_ns) {
                     *abort_flag = 1;
+                    ptx::griddep_wait();
                     if (atomicCAS(&prm.status[0], 0, TILEMIX_ERR_DEVICE_TIMEOUT) == 0) {
                         prm.status[1] = 16; prm.status[2] = t0; prm.status[3] = which;
                     }
