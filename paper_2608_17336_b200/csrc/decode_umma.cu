@@ -382,10 +382,11 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         // the fixed cost of its waits and its proxy fence: two groups in parallel halve it per tile).  A thread takes
         // its two 16-byte pieces of a landed V8 tile into registers (the ring unit goes back to the producer at
         // once) and converts them when the PV that read the buffer last has retired.
-        // Piece idx of a half = columns 16q .. 16q+15 of one of its 64 keys.  Eight consecutive pieces are the four
-        // pieces of one 64-column half of two adjacent keys: as FP16 they are the even 16-byte chunks of one key's
-        // 128-byte row and the odd ones of the other's (the swizzle flips the parity with the row), so a quarter
-        // warp's 128-bit stores fall into eight different bank groups.
+        // Piece idx of a half = columns 16q .. 16q+15 of one of its 64 keys.  Eight consecutive pieces are four
+        // pieces of one 64-column half of a key and four of the other half of the next key: read as INT8 they are
+        // the two halves of a 128-byte line, and as FP16 they are the even 16-byte chunks of one key's 128-byte row
+        // and the odd ones of the other's (the swizzle flips the parity with the row), so a quarter warp's
+        // 128-bit loads and stores each fall into eight different bank groups.
         const int hf = (warp - kConvWarp0) >> 3;
         const int cid = ((warp - kConvWarp0) & 7) * 32 + lane;
         constexpr int kGroupThreads = kConvThreads / 2, kPer = (T / 2) * D / 16 / kGroupThreads;
@@ -400,7 +401,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
                 const int idx = cid + kGroupThreads * j;
-                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = (((idx >> 3) & 1) << 2) | (idx & 3);
+                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = ((((idx >> 3) ^ (idx >> 2)) & 1) << 2) | (idx & 3);
                 in[j] = *reinterpret_cast<const uint4*>(src + row * D + q * 16);
             }
             __syncwarp();
@@ -409,7 +410,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
 #pragma unroll
             for (int j = 0; j < kPer; ++j) {
                 const int idx = cid + kGroupThreads * j;
-                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = (((idx >> 3) & 1) << 2) | (idx & 3);
+                const int row = ((idx >> 4) << 1) | ((idx >> 2) & 1), q = ((((idx >> 3) ^ (idx >> 2)) & 1) << 2) | (idx & 3);
                 const uint32_t w[4] = {in[j].x, in[j].y, in[j].z, in[j].w};
                 uint32_t h[8];
 #pragma unroll
