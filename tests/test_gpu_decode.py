@@ -169,3 +169,30 @@ def test_decode_without_fp16_cache_reports_an_fp16_routed_group():
     res = tm.tilemix_decode_int8kv(p, q.to(dev), None, k8, ks, v8, vs, words,
                                    torch.from_numpy(np.asarray([640, 300], np.int32)).to(dev))
     assert tm.tilemix_read_status(res["workspace"])[0] == 0
+
+
+@pytest.mark.parametrize("n_splits", [1, 2])
+def test_decode_running_maximum_moves_many_times(n_splits):
+    """Scores that climb along the cache (about 2 log2 units per 128-key tile, far more than the 2^8 by which the
+    lazy running maximum may lag): the maximum moves every few steps, in every split and stream, so the rescale of
+    the row sums and of the accumulated output (in tensor memory in the tcgen05 form of the step) is exercised many
+    times.  The same cache read backwards (maximum first) must work too."""
+    B, Hq, Hk, L, d, tile, G = 2, 8, 2, 3000, 128, 128, 1
+    q, k, v, route, lens = _case(B, Hq, Hk, L, d, tile, G, seed=51, lens=[3000, 2500], f8=0.5)
+    rep = Hq // Hk
+    qm = q.float().view(B, Hk, rep, d).mean(2)                       # a direction every head of the group likes
+    qm = qm / qm.norm(dim=-1, keepdim=True)
+    ramp = torch.linspace(0.0, 1.0, L).view(1, 1, L, 1)
+    for sign in (1.0, -1.0):
+        kk = (0.3 * k.float() + sign * 60.0 * ramp * qm.unsqueeze(2)).half()
+        # the ramp is what the test is about: the scores of every head span far more than 2^8
+        s = torch.einsum("bhrd,bhld->bhrl", q.float().view(B, Hk, rep, d), kk.float()) * (1.4427 / d ** 0.5)
+        assert (s.max(-1).values - s.min(-1).values).min() > 30.0
+        _check(q, kk, v, route, lens, tile, G, n_splits=n_splits)
+
+
+def test_decode_more_tiles_per_split_than_the_staged_metadata():
+    """A split of 266 key tiles: the step stages route bit and block scales of its first 256 tiles in shared memory and
+    takes the rest from global memory; more than 32 routing groups per row, so more than one mask word."""
+    q, k, v, route, lens = _case(1, 4, 1, 34000, 128, 128, 3, seed=52, lens=[33990], f8=0.5)
+    _check(q, k, v, route, lens, 128, 3, n_splits=1)
