@@ -145,6 +145,30 @@ int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, cons
                                 const uint32_t* mask_words, void* out_f16, float* lse, void* workspace,
                                 size_t workspace_bytes, const tilemix_debug_t* dbg, void* stream);
 
+/* Chunked prefill against an INT8 VALUE cache (App. C, "Additional Execution Interfaces": cached V8 is
+ * converted to FP16 on chip and its block scale is folded into the probability tile before the PV product).
+ * As tilemix_attention_fwd_chunk, but the values are INT8 with one FP32 scale per block of tile_n tokens
+ * (the cache layout of tilemix_decode_int8kv):
+ *   o_i = sum_j softmax(s_i)_j * delta_V[blk(j)] * v8_j  over the keys j <= kv_len - p->seqlen + i,
+ * computed as P' V with P'_ij = FP16(softmax numerator * delta_V[blk(j)]) and V the exact FP16 image of V8,
+ * FP32 accumulation (the row sum is of the unscaled numerators).  The scores are those of
+ * tilemix_attention_fwd_chunk (routed FP16 / INT8 QK^T).  With kv_len == p->seqlen it is a prefill that writes
+ * against a freshly quantised value cache; with p->seqlen == tile it is one tile of new queries.
+ *   v_i8     INT8 [B,Hk,kv_len,d], dense;  v_scale FP32 [B,Hk,ceil(kv_len/tile_n)]
+ *   workspace  tilemix_chunk_v8_workspace_size(p, kv_len) bytes: the status record and an FP16 image of the value
+ *            cache.  The conversion is a kernel of its own in front of the attention kernel (two launches): the
+ *            image passes through device memory once per call (3 bytes per cached element, ~1 % of the attention
+ *            kernel's time at a 4096-token chunk of a 32K context) instead of being made tile by tile in shared
+ *            memory; the arithmetic is the same.
+ * Dense batches, quantise-once operands (no TILEMIX_QUANT_ON_THE_FLY); the v_stride of `p` is ignored.
+ * Everything else as for tilemix_attention_fwd_chunk. */
+size_t tilemix_chunk_v8_workspace_size(const tilemix_problem_t* p, int32_t kv_len);
+int tilemix_attention_fwd_chunk_v8(const tilemix_problem_t* p, int32_t kv_len, const void* q_f16,
+                                   const void* k_f16, const int8_t* v_i8, const float* v_scale,
+                                   const int8_t* q_i8, const int8_t* k_i8, const float* q_scale,
+                                   const float* k_scale, const uint32_t* mask_words, void* out_f16,
+                                   float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Same computation as tilemix_attention_fwd for callers that cannot hand it a workspace because
  * they cannot allocate device memory at all: a process whose whole GPU memory was claimed at
  * start-up by another allocator or memory pool (any later cudaMalloc fails), or a code path that

@@ -75,3 +75,52 @@ def decode(q16, k16, k8, k_scale, v8, v_scale, words, cache_len, tile_n, group, 
             out[b, hq] = (p[:, None] * v).sum(0) / z
             lse[b, hq] = m + np.log(z)
     return out, lse
+
+
+def chunk_v8(q16, q8, q_scale, k16, k8, k_scale, v8, v_scale, words, tile, group, blk_q=0, blk_k=0,
+             softmax_scale=0.0):
+    """Chunked prefill against an INT8 value cache (App. C, "Additional Execution Interfaces"; Sec. 3.1 softmax;
+    App. C score formulas), the definition written out: the queries are the LAST L_q tokens of a context of L_k
+    tokens, query i sits at context position c = L_k - L_q + i and attends to the keys j <= c;
+
+      INT8-routed group:  s_ij = delta_q[blk_q(i)] * delta_K[blk_k(j)] * (q8_i . k8_j) * scale
+      FP16-routed group:  s_ij = (q_i . k16_j) * scale
+      o_i = sum_j softmax(s_i)_j * delta_V[j // tile] * v8_j
+
+    where bit g of the mask row of (h_k, query tile c // tile) routes the keys [g*G*tile, (g+1)*G*tile).
+    q16 uint16 / q8 int8 [B,Hq,Lq,d]; q_scale float32 [B,Hq,ceil(Lq/blk_q)]; k16 uint16 / k8, v8 int8 [B,Hk,Lk,d];
+    k_scale float32 [B,Hk,ceil(Lk/blk_k)]; v_scale float32 [B,Hk,ceil(Lk/tile)]; words uint32 [nb,Hk,ceil(Lk/tile),W]
+    (the words of the whole context).  Returns (out float64 [B,Hq,Lq,d], lse float64 [B,Hq,Lq])."""
+    B, Hq, Lq, d = q16.shape
+    Hk, Lk = k8.shape[1], k8.shape[2]
+    rep = Hq // Hk
+    blk_q = blk_q or tile
+    blk_k = blk_k or tile
+    off = Lk - Lq
+    scale = softmax_scale if softmax_scale > 0 else 1.0 / np.sqrt(d)
+    q = half_bits_to_f64(q16)
+    j = np.arange(Lk)
+    grp = j // (tile * group)
+    out = np.zeros((B, Hq, Lq, d))
+    lse = np.zeros((B, Hq, Lq))
+    for b in range(B):
+        for hq in range(Hq):
+            hk = hq // rep
+            k = half_bits_to_f64(k16[b, hk])
+            v = v8[b, hk].astype(np.float64) * v_scale[b, hk, j // tile].astype(np.float64)[:, None]
+            dots8 = q8[b, hq].astype(np.int64) @ k8[b, hk].astype(np.int64).T                      # [Lq, Lk], exact
+            dq = q_scale[b, hq, np.arange(Lq) // blk_q].astype(np.float64)[:, None]
+            dk = k_scale[b, hk, j // blk_k].astype(np.float64)[None, :]
+            s8 = dq * dk * dots8 * scale
+            s16 = (q[b, hq] @ k.T) * scale
+            for i in range(Lq):
+                c = off + i
+                wrow = words[0 if words.shape[0] == 1 else b, hk, c // tile]
+                bit = ((wrow[grp[:c + 1] >> 5] >> (grp[:c + 1] & 31).astype(np.uint32)) & 1).astype(bool)
+                s = np.where(bit, s8[i, :c + 1], s16[i, :c + 1])
+                m = s.max()
+                p = np.exp(s - m)
+                z = p.sum()
+                out[b, hq, i] = (p[:, None] * v[:c + 1]).sum(0) / z
+                lse[b, hq, i] = m + np.log(z)
+    return out, lse

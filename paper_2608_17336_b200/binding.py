@@ -25,6 +25,7 @@ EXPORTS = (
     "tilemix_varlen_counts", "tilemix_varlen_workspace_size", "tilemix_quantize_qk_varlen",
     "tilemix_pack_routing_mask_varlen", "tilemix_attention_fwd_varlen",
     "tilemix_decode_workspace_size", "tilemix_decode_int8kv", "tilemix_attention_fwd_chunk",
+    "tilemix_chunk_v8_workspace_size", "tilemix_attention_fwd_chunk_v8",
     "tilemix_test_drop_copy", "tilemix_tensor_peak_probe",
 )
 
@@ -96,6 +97,10 @@ def lib() -> ctypes.CDLL:
                                             ctypes.POINTER(DebugStruct), vp]
         L.tilemix_attention_fwd_chunk.argtypes = [pp, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                                   ctypes.c_size_t, ctypes.POINTER(DebugStruct), vp]
+        L.tilemix_chunk_v8_workspace_size.argtypes = [pp, ctypes.c_int32]
+        L.tilemix_chunk_v8_workspace_size.restype = ctypes.c_size_t
+        L.tilemix_attention_fwd_chunk_v8.argtypes = [pp, ctypes.c_int32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                     ctypes.c_size_t, vp]
         L.tilemix_attention_fwd_noalloc.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                                     ctypes.POINTER(DebugStruct), ctypes.POINTER(vp), vp]
         L.tilemix_prefill_host.argtypes = [pp, vp, vp, vp, vp, u32, vp, vp, ctypes.c_size_t, vp]
@@ -423,4 +428,26 @@ def tilemix_attention_fwd_chunk(p: ProblemStruct, kv_len: int, q, k, v, q8, k8, 
                                            _ptr(q_scale), _ptr(k_scale), _ptr(words), _ptr(out), _ptr(lse),
                                            _ptr(workspace), workspace.numel(), None, _stream())
     _check(rc, "tilemix_attention_fwd_chunk")
+    return {"out": out, "lse": lse, "workspace": workspace}
+
+
+def tilemix_chunk_v8_workspace_size(p: ProblemStruct, kv_len: int) -> int:
+    return int(lib().tilemix_chunk_v8_workspace_size(ctypes.byref(p), kv_len))
+
+
+def tilemix_attention_fwd_chunk_v8(p: ProblemStruct, kv_len: int, q, k, v8, v_scale, q8, k8, q_scale, k_scale, words,
+                                   out=None, want_lse=False, workspace=None):
+    """As tilemix_attention_fwd_chunk with the values taken from an INT8 cache: v8 int8 [B,Hk,kv_len,d] (dense),
+    v_scale float32 [B,Hk,ceil(kv_len/tile)]."""
+    dev = q.device
+    if out is None:
+        out = torch.empty((p.batch, p.heads_q, p.seqlen, p.head_dim), dtype=torch.float16, device=dev)
+    lse = torch.empty((p.batch, p.heads_q, p.seqlen), dtype=torch.float32, device=dev) if want_lse else None
+    pp = _with_strides(p, q=q, k=k, o=out)
+    if workspace is None:
+        workspace = torch.empty(max(tilemix_chunk_v8_workspace_size(pp, kv_len), 4096), dtype=torch.uint8, device=dev)
+    rc = lib().tilemix_attention_fwd_chunk_v8(ctypes.byref(pp), kv_len, _ptr(q), _ptr(k), _ptr(v8), _ptr(v_scale),
+                                              _ptr(q8), _ptr(k8), _ptr(q_scale), _ptr(k_scale), _ptr(words), _ptr(out),
+                                              _ptr(lse), _ptr(workspace), workspace.numel(), _stream())
+    _check(rc, "tilemix_attention_fwd_chunk_v8")
     return {"out": out, "lse": lse, "workspace": workspace}

@@ -1,4 +1,5 @@
 // C ABI of libtilemix: argument validation on the host, then the kernel launchers.
+#include <cuda_fp16.h>
 #include <math.h>
 #include <string.h>
 
@@ -54,7 +55,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 int checked_attention(const Geometry& g, const void* q_f16, const void* k_f16, const void* v_f16, const int8_t* q_i8,
                       const int8_t* k_i8, const float* q_scale, const float* k_scale, const uint32_t* mask_words,
                       void* out_f16, float* lse, void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg,
-                      void* stream) {
+                      void* stream, const float* v_scale = nullptr) {
     if (!q_f16 || !k_f16 || !v_f16 || !out_f16 || !workspace) return TILEMIX_ERR_NULL;
     const bool force16 = (g.flags & TILEMIX_FORCE_FP16) != 0;
     const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;   // INT8 operands and scales are made on chip
@@ -78,7 +79,50 @@ int checked_attention(const Geometry& g, const void* q_f16, const void* k_f16, c
     const int rc = check_device();
     if (rc) return rc;
     return launch_attention(g, q_f16, k_f16, v_f16, force16 ? nullptr : q_i8, force16 ? nullptr : k_i8, q_scale,
-                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream));
+                            k_scale, mask_words, out_f16, lse, workspace, dbg, static_cast<cudaStream_t>(stream),
+                            nullptr, 0, v_scale);
+}
+
+// INT8 value cache -> its exact FP16 image (|x| <= 127 is exact in binary16), 16 values per thread.
+__global__ void v8_to_f16_kernel(const int8_t* __restrict__ v8, __half* __restrict__ v16, int64_t n16) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n16) return;
+    const uint4 in = reinterpret_cast<const uint4*>(v8)[i];
+    const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+    uint32_t h[8];
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int lo = static_cast<int8_t>(w[y] >> (16 * e)), hi = static_cast<int8_t>(w[y] >> (16 * e + 8));
+            const __half2 v = __floats2half2_rn(static_cast<float>(lo), static_cast<float>(hi));
+            h[2 * y + e] = *reinterpret_cast<const uint32_t*>(&v);
+        }
+    }
+    uint4* out = reinterpret_cast<uint4*>(v16) + 2 * i;
+    out[0] = make_uint4(h[0], h[1], h[2], h[3]);
+    out[1] = make_uint4(h[4], h[5], h[6], h[7]);
+}
+
+// Geometry of a chunk of the last p->seqlen tokens of a kv_len-token context (K and V are kv_len tokens long).
+int resolve_chunk(const tilemix_problem_t* p, int32_t kv_len, Geometry* g) {
+    if (p == nullptr) return TILEMIX_ERR_NULL;
+    if (kv_len < p->seqlen || p->tile_m <= 0 || p->tile_m != p->tile_n || (kv_len - p->seqlen) % p->tile_m != 0)
+        return TILEMIX_ERR_SHAPE;
+    // K and V are kv_len tokens long: dense strides are theirs, not the chunk's
+    tilemix_problem_t q = *p;
+    if (all_zero(q.k_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.k_stride);
+    if (all_zero(q.v_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.v_stride);
+    const int rc = resolve(&q, g);
+    if (rc) return rc;
+    g->Lk = kv_len;
+    g->kv_off = (kv_len - g->L) / g->tile_m;
+    g->T_n = static_cast<int>(ceil_div(kv_len, g->tile_n));
+    g->mask_T_m = g->T_n;                      // the mask words of the whole context
+    g->ks_blocks = static_cast<int>(ceil_div(kv_len, g->blk_k));
+    g->T_mask = static_cast<int>(ceil_div(kv_len, static_cast<int64_t>(g->G) * g->tile_n));
+    g->W = static_cast<int>(ceil_div(g->T_mask, 32));
+    return TILEMIX_OK;
 }
 
 }  // namespace
@@ -160,25 +204,45 @@ int tilemix_attention_fwd_chunk(const tilemix_problem_t* p, int32_t kv_len, cons
                                 const void* v_f16, const int8_t* q_i8, const int8_t* k_i8, const float* q_scale,
                                 const float* k_scale, const uint32_t* mask_words, void* out_f16, float* lse,
                                 void* workspace, size_t workspace_bytes, const tilemix_debug_t* dbg, void* stream) {
-    if (p == nullptr) return TILEMIX_ERR_NULL;
-    if (kv_len < p->seqlen || p->tile_m <= 0 || p->tile_m != p->tile_n || (kv_len - p->seqlen) % p->tile_m != 0)
-        return TILEMIX_ERR_SHAPE;
-    // K and V are kv_len tokens long: dense strides are theirs, not the chunk's
-    tilemix_problem_t q = *p;
-    if (all_zero(q.k_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.k_stride);
-    if (all_zero(q.v_stride)) dense_strides(q.heads_kv, kv_len, q.head_dim, q.v_stride);
     Geometry g;
-    int rc = resolve(&q, &g);
+    const int rc = resolve_chunk(p, kv_len, &g);
     if (rc) return rc;
-    g.Lk = kv_len;
-    g.kv_off = (kv_len - g.L) / g.tile_m;
-    g.T_n = static_cast<int>(ceil_div(kv_len, g.tile_n));
-    g.mask_T_m = g.T_n;                      // the mask words of the whole context
-    g.ks_blocks = static_cast<int>(ceil_div(kv_len, g.blk_k));
-    g.T_mask = static_cast<int>(ceil_div(kv_len, static_cast<int64_t>(g.G) * g.tile_n));
-    g.W = static_cast<int>(ceil_div(g.T_mask, 32));
     return checked_attention(g, q_f16, k_f16, v_f16, q_i8, k_i8, q_scale, k_scale, mask_words, out_f16, lse, workspace,
                              workspace_bytes, dbg, stream);
+}
+
+size_t tilemix_chunk_v8_workspace_size(const tilemix_problem_t* p, int32_t kv_len) {
+    Geometry g;
+    if (resolve_chunk(p, kv_len, &g)) return 0;
+    return kStatusAreaBytes + static_cast<size_t>(g.B) * g.Hk * g.Lk * g.d * sizeof(__half);
+}
+
+int tilemix_attention_fwd_chunk_v8(const tilemix_problem_t* p, int32_t kv_len, const void* q_f16, const void* k_f16,
+                                   const int8_t* v_i8, const float* v_scale, const int8_t* q_i8, const int8_t* k_i8,
+                                   const float* q_scale, const float* k_scale, const uint32_t* mask_words,
+                                   void* out_f16, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+    if (p == nullptr) return TILEMIX_ERR_NULL;
+    tilemix_problem_t q = *p;
+    for (int i = 0; i < 3; ++i) q.v_stride[i] = 0;     // the INT8 value cache is dense; so is its FP16 image
+    Geometry g;
+    int rc = resolve_chunk(&q, kv_len, &g);
+    if (rc) return rc;
+    if (!v_i8 || !v_scale || !workspace) return TILEMIX_ERR_NULL;
+    if (g.flags & TILEMIX_QUANT_ON_THE_FLY) return TILEMIX_ERR_UNSUPPORTED;
+    if (!aligned16(v_i8) || !aligned16(workspace)) return TILEMIX_ERR_ALIGN;
+    const size_t n = static_cast<size_t>(g.B) * g.Hk * g.Lk * g.d;
+    if (workspace_bytes < kStatusAreaBytes + n * sizeof(__half)) return TILEMIX_ERR_WORKSPACE;
+    if ((rc = check_device())) return rc;
+    __half* v16 = reinterpret_cast<__half*>(static_cast<uint8_t*>(workspace) + kStatusAreaBytes);
+    const int64_t n16 = static_cast<int64_t>(n / 16);  // head_dim is 64 or 128: whole 16-byte pieces
+    if (n16 > 0) {
+        v8_to_f16_kernel<<<static_cast<unsigned>((n16 + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(v_i8, v16, n16);
+        g_launch_count.fetch_add(1);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return static_cast<int>(e);
+    }
+    return checked_attention(g, q_f16, k_f16, v16, q_i8, k_i8, q_scale, k_scale, mask_words, out_f16, lse, workspace,
+                             kStatusAreaBytes, nullptr, stream, v_scale);
 }
 
 int tilemix_mask_words_per_row(int seqlen, int tile_n, int group) {

@@ -116,6 +116,8 @@ struct Params {
     float scale_log2;             // softmax scale * log2(e)
     const float* q_scale;         // [B,Hq,T_m]; variable-length batch: [sum T_m, Hq]
     const float* k_scale;         // [B,Hk,T_n]; variable-length batch: [sum T_n, Hk]
+    const float* v_scale;         // [B,Hk,vs_blocks] block scales of an INT8 value cache (VS instances), else null
+    int vs_blocks;                // key tiles of the context
     const uint32_t* words;        // [nb,Hk,T_m,W] or null (all FP16)
     // Variable-length batch (null = one dense batch): prefix sums over the sequences.  Then B = 1,
     // L = total tokens and T_m = total query-tile rows of the packed batch.
@@ -187,7 +189,7 @@ struct Ring {
 // OTF: on-the-fly operand generation (App. D, "fused on-the-fly" mode): there are no INT8 copies of Q and K
 // and no scales in global memory; a quantiser warp makes them in shared memory from the FP16 tiles, for
 // the key tiles some query tile of the CTA routes to INT8 only.
-template <int D, int T, bool VL, bool OTF>
+template <int D, int T, bool VL, bool OTF, bool VS = false>
 __global__ void __launch_bounds__(OTF ? kThreadsOtf : kThreads, 1)
 attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                  const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16,
@@ -733,6 +735,10 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             const bool k_half = prm.k_half_blocks != 0;
             auto load_dk = [&](int blk) { return (prm.has_int8 && !OTF && blk < n_kblk) ? dk_row[blk * dk_step] : 0.f; };
             float dk_cur = 0.f, dk_next = load_dk(0);
+            // VS: delta_V of the key tile (block = key tile) of the INT8 value cache the FP16 V operand was made from
+            const float* dv_row = nullptr;
+            if constexpr (VS) dv_row = prm.v_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.vs_blocks;
+            float dv = 1.f;
             float a = prm.scale_log2;
             uint32_t int8_route = 0u;
             const int n_steps = 2 * (k_t + 1);
@@ -742,6 +748,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
             for (int u = 0; u < n_steps; ++u) {
                 const int j = u >> 1, h = u & 1;
                 if (h == 0) int8_route = (sched(j) >> t) & 1u;
+                if constexpr (VS) { if (h == 0) dv = dv_row[j]; }
                 if (h == 0 || k_half) {
                     dk_cur = dk_next;
                     dk_next = load_dk(k_half ? u + 1 : j + 1);
@@ -781,18 +788,18 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 float alpha[2] = {1.f, 1.f}, sum[2] = {0.f, 0.f};
                 bool grow = false;
                 uint32_t p[2 * NB];
-                ptx::tmem_wait_ld();
+                ptx::tmem_wait_ld_dep(s);     // ties the registers to the wait: no use of them moves above it
                 if (!redo) {
                     if (!int8_route) {
                         const float addend[2] = {-m_run[0], -m_run[1]};
-                        softmax_step_fast<NB, kFp32>(s, a, addend, p, sum);
+                        softmax_step_fast<NB, kFp32, VS>(s, a, addend, p, sum, dv);
                     } else if (a * kInt8Bias <= kFoldLimit) {
                         // one explicit FMA: every instantiation of the kernel rounds the addend the same way
                         const float addend[2] = {-__fmaf_rn(a, kInt8Bias, m_run[0]), -__fmaf_rn(a, kInt8Bias, m_run[1])};
-                        softmax_step_fast<NB, kInt8Folded>(s, a, addend, p, sum);
+                        softmax_step_fast<NB, kInt8Folded, VS>(s, a, addend, p, sum, dv);
                     } else {
                         const float addend[2] = {-m_run[0], -m_run[1]};
-                        softmax_step_fast<NB, kInt8Exact>(s, a, addend, p, sum);
+                        softmax_step_fast<NB, kInt8Exact, VS>(s, a, addend, p, sum, dv);
                     }
                     redo = __any_sync(0xffffffffu, !(sum[0] <= exp2f(kAccept) && sum[1] <= exp2f(kAccept)));   // also true for a NaN
                 }
@@ -857,7 +864,8 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                                                          a2, make_float2(-m_run[k], -m_run[k]));
                             const float2 pp = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
                             acc[k] = __fadd2_rn(acc[k], pp);
-                            p[2 * i + k] = pack_half2(pp.x, pp.y);
+                            if constexpr (VS) p[2 * i + k] = pack_half2(pp.x * dv, pp.y * dv);
+                            else p[2 * i + k] = pack_half2(pp.x, pp.y);
                         }
                     }
                     sum[0] = acc[0].x + acc[0].y;
@@ -881,7 +889,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[16];
                         ptx::tmem_ld16x256_x4(t_o + c * 32, o);
-                        ptx::tmem_wait_ld();
+                        ptx::tmem_wait_ld_dep(o);
 #pragma unroll
                         for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha[(e >> 1) & 1]);
                         ptx::tmem_st16x256_x4(t_o + c * 32, o);
@@ -916,7 +924,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[16];
                     ptx::tmem_ld16x256_x4(t_o + c * 32, o);
-                    ptx::tmem_wait_ld();
+                    ptx::tmem_wait_ld_dep(o);
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
                         if (z[k] == 0.f) continue;     // a row beyond the sequence (or the 64-row tile): not written
@@ -978,13 +986,14 @@ template <int D, int T>
 int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, const int8_t* q8,
                 const int8_t* k8, const float* qs, const float* ks, const uint32_t* words, void* out,
                 float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream,
-                const VarlenDev* vl, int total_pairs) {
+                const VarlenDev* vl, int total_pairs, const float* v_scale) {
     using C = Cfg<D, T>;
     EncodeTiledFn enc = nullptr;
     int rc = get_encoder(&enc);
     if (rc) return rc;
     const bool otf = (g.flags & TILEMIX_QUANT_ON_THE_FLY) != 0;
     if (otf && (vl != nullptr || !(D == 128 && T == 128) || g.blk_k != g.tile_n)) return TILEMIX_ERR_UNSUPPORTED;
+    if (v_scale != nullptr && (otf || vl != nullptr)) return TILEMIX_ERR_UNSUPPORTED;   // value-cache scales: dense, quantise-once
     const bool has8 = !(g.flags & TILEMIX_FORCE_FP16) && (q8 != nullptr || otf);
     CUtensorMap tq, tk, tv, tq8, tk8;
     if ((rc = encode_map(enc, &tq, q, 2, g.d, g.L, g.Hq, g.B, g.qs, 64, C::kM, CU_TENSOR_MAP_SWIZZLE_128B))) return rc;
@@ -1019,6 +1028,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     prm.has_int8 = has8 ? 1 : 0;
     prm.scale_log2 = g.scale * kLog2e;
     prm.q_scale = qs; prm.k_scale = ks;
+    prm.v_scale = v_scale; prm.vs_blocks = g.T_n;
     prm.words = has8 ? words : nullptr;
     prm.out = static_cast<__half*>(out);
     prm.os[0] = g.os[0]; prm.os[1] = g.os[1]; prm.os[2] = g.os[2];
@@ -1037,6 +1047,7 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     if constexpr (D == 128 && T == 128) {
         if (otf) kernel = attention_kernel<D, T, false, true>;
     }
+    if (v_scale != nullptr) kernel = attention_kernel<D, T, false, false, true>;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
     if (e != cudaSuccess) return static_cast<int>(e);
     const int64_t ctas = vl ? static_cast<int64_t>(g.Hq) * total_pairs
@@ -1059,13 +1070,13 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
 int launch_attention(const Geometry& g, const void* q, const void* k, const void* v, const int8_t* q8,
                      const int8_t* k8, const float* qs, const float* ks, const uint32_t* words, void* out,
                      float* lse, void* workspace, const tilemix_debug_t* dbg, cudaStream_t stream,
-                     const VarlenDev* vl, int total_pairs) {
+                     const VarlenDev* vl, int total_pairs, const float* v_scale) {
     if (g.d == 128 && g.tile_m == 128)
         return launch_impl<128, 128>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream, vl,
-                                     total_pairs);
+                                     total_pairs, v_scale);
     if (g.d == 64 && g.tile_m == 64)
         return launch_impl<64, 64>(g, q, k, v, q8, k8, qs, ks, words, out, lse, workspace, dbg, stream, vl,
-                                   total_pairs);
+                                   total_pairs, v_scale);
     return TILEMIX_ERR_UNSUPPORTED;
 }
 

@@ -92,6 +92,8 @@ int launch_attention(const Geometry& g, const void* q, const void* k, const void
                      const int8_t* q8, const int8_t* k8, const float* qs, const float* ks,
                      const uint32_t* words, void* out, float* lse, void* workspace,
                      const tilemix_debug_t* dbg, cudaStream_t stream, const VarlenDev* vl = nullptr,
-                     int total_pairs = 0);
+                     int total_pairs = 0, const float* v_scale = nullptr);
+// `v_scale` (nullable; dense batches only): `v` is the exact FP16 image of an INT8 value cache and the block scale
+// of key tile j is folded into the probabilities of that tile before they are rounded to FP16.
 
 }  // namespace tilemix

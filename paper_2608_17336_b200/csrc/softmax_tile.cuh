@@ -53,10 +53,11 @@ constexpr float kInt8Bias = 12582912.f;   // 1.5 * 2^23
 // One interior step (NB blocks of 8 key columns, no causal mask) in one pass with the current running
 // maxima: raw accumulators s -> P = 2^(a*raw - m) rounded to FP16 (p[2i + k] = the pair of row k in block
 // i) and this thread's part of the FP32 row sums.  addend[k] = -m_k (kFp32, kInt8Exact) or -(m_k + a*1.5*2^23)
-// (kInt8Folded).
-template <int NB, int KIND>
+// (kInt8Folded).  VS: the probabilities are multiplied by `dv` (the block scale of an INT8 value cache, App. C:
+// folded into the probability tile) before they are rounded to FP16; the row sums are of the unscaled values.
+template <int NB, int KIND, bool VS = false>
 __device__ __forceinline__ void softmax_step_fast(const uint32_t (&s)[4 * NB], float a, const float (&addend)[2],
-                                                  uint32_t (&p)[2 * NB], float (&sum)[2]) {
+                                                  uint32_t (&p)[2 * NB], float (&sum)[2], float dv = 1.f) {
     const float2 a2 = make_float2(a, a);
     const float2 unbias = make_float2(-kInt8Bias, -kInt8Bias);
     float2 acc[2] = {{0.f, 0.f}, {0.f, 0.f}};
@@ -75,7 +76,12 @@ __device__ __forceinline__ void softmax_step_fast(const uint32_t (&s)[4 * NB], f
             const float2 t2 = __ffma2_rn(x, a2, make_float2(addend[k], addend[k]));
             const float2 e = make_float2(fast_exp2(t2.x), fast_exp2(t2.y));
             acc[k] = __fadd2_rn(acc[k], e);
-            p[2 * i + k] = pack_half2(e.x, e.y);
+            if constexpr (VS) {
+                const float2 ev = __fmul2_rn(e, make_float2(dv, dv));
+                p[2 * i + k] = pack_half2(ev.x, ev.y);
+            } else {
+                p[2 * i + k] = pack_half2(e.x, e.y);
+            }
         }
     }
     sum[0] = acc[0].x + acc[0].y;

@@ -215,3 +215,27 @@ def test_decode_host_side_validation(lib):
     assert call(ok, k16=None, words=None) == b.ERR_NULL                               # all FP16 without an FP16 cache
     assert call(ok, k8=ctypes.c_void_p(4100)) == b.ERR_ALIGN
     assert call(ok, nbytes=size - 1) == b.ERR_WORKSPACE
+
+
+def test_chunk_v8_host_side_validation(lib):
+    """tilemix_attention_fwd_chunk_v8: what the host can refuse before any launch."""
+    one = ctypes.c_void_p(0x1000)
+    p = b.problem(1, 4, 2, 256, 128, 128, 128)
+    need = lib.tilemix_chunk_v8_workspace_size(ctypes.byref(p), 1024)
+    assert need == 4096 + 1 * 2 * 1024 * 128 * 2                       # status record + FP16 image of the value cache
+    assert lib.tilemix_chunk_v8_workspace_size(ctypes.byref(p), 1000) == 0          # offset not a multiple of the tile
+    args = [one] * 11                                                  # q, k, v8, v_scale, q8, k8, qs, ks, words, out, lse
+    call = lambda prob, kv, a, ws=one, nbytes=need: lib.tilemix_attention_fwd_chunk_v8(
+        ctypes.byref(prob), kv, *a, ws, nbytes, None)
+    assert call(p, 1000, args) == b.ERR_SHAPE
+    assert call(p, 128, args) == b.ERR_SHAPE                           # context shorter than the chunk
+    no_scale = list(args); no_scale[3] = None
+    assert call(p, 1024, no_scale) == b.ERR_NULL
+    no_v = list(args); no_v[2] = None
+    assert call(p, 1024, no_v) == b.ERR_NULL
+    assert call(p, 1024, args, nbytes=need - 1) == b.ERR_WORKSPACE
+    skew = list(args); skew[2] = ctypes.c_void_p(0x1008)
+    assert call(p, 1024, skew) == b.ERR_ALIGN
+    otf = b.problem(1, 4, 2, 256, 128, 128, 128, flags=b.QUANT_ON_THE_FLY)
+    assert call(otf, 1024, args) == b.ERR_UNSUPPORTED
+    assert lib.tilemix_attention_fwd_chunk_v8(None, 1024, *args, one, need, None) == b.ERR_NULL

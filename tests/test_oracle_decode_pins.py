@@ -177,3 +177,95 @@ def test_per_batch_mask_rows_select_their_own_batch_entry():
     for e in range(0, d, 7):
         o = sum(w[j] * float(c["vs"][b, hk, j // tile]) * int(c["v8"][b, hk, j, e]) for j in range(131)) / sum(w)
         assert abs(o - out[b, hq, e]) < 1e-12
+
+
+# ---- chunked prefill against an INT8 value cache (chunk_v8) -------------------------------------------------------
+
+def _chunk_case(B, Hq, Hk, Lk, Lq, d, tile, G, seed, f8=0.5, pow2_v=False, blk_q=0):
+    rng = np.random.default_rng(seed)
+    Q = rng.standard_normal((B, Hq, Lk, d)).astype(np.float16)          # the whole context's queries; the chunk = last Lq
+    k = rng.standard_normal((B, Hk, Lk, d)).astype(np.float16)
+    v = rng.standard_normal((B, Hk, Lk, d)).astype(np.float16)
+    q16 = np.ascontiguousarray(Q.view(np.uint16)); k16 = np.ascontiguousarray(k.view(np.uint16))
+    q8, qs = oracle.quantize(q16, blk_q or tile)
+    k8, ks = oracle.quantize(k16, tile)
+    if pow2_v:
+        v8 = rng.integers(-127, 128, (B, Hk, Lk, d)).astype(np.int8)
+        vs = (2.0 ** rng.integers(-6, -2, (B, Hk, -(-Lk // tile)))).astype(np.float32)
+    else:
+        v8, vs = oracle.quantize(np.ascontiguousarray(v.view(np.uint16)), tile)
+    p = oracle.Problem(B, Hq, Hk, Lk, d, tile, tile, G, blk_q=blk_q)
+    route = (rng.random((1, Hk, p.T_m, p.T_mask)) < f8).astype(np.uint8)
+    words, _ = oracle.pack(p, route)
+    off = Lk - Lq
+    bq = blk_q or tile
+    chunk = dict(q16=np.ascontiguousarray(q16[:, :, off:]), q8=np.ascontiguousarray(q8[:, :, off:]),
+                 qs=np.ascontiguousarray(qs[:, :, off // bq:]))
+    return dict(p=p, q16=q16, q8=q8, qs=qs, k16=k16, k8=k8, ks=ks, v8=v8, vs=vs, route=route, words=words, off=off,
+                chunk=chunk, tile=tile, G=G, blk_q=blk_q)
+
+
+def _chunk_run(c):
+    ch = c["chunk"]
+    return od.chunk_v8(ch["q16"], ch["q8"], ch["qs"], c["k16"], c["k8"], c["ks"], c["v8"], c["vs"], c["words"],
+                       c["tile"], c["G"], blk_q=c["blk_q"])
+
+
+def test_chunk_v8_with_a_lossless_value_cache_equals_the_prefill_oracle_rows():
+    """Power-of-two block scales make delta_V * V8 exactly representable in FP16: the chunk against the INT8 value
+    cache must then equal the already pinned prefill oracle on the same rows of the whole context (GQA, grouping
+    factor 2, mixed routes, a ragged last tile)."""
+    B, Hq, Hk, Lk, Lq, d, tile, G = 2, 4, 2, 300, 172, 32, 64, 2
+    c = _chunk_case(B, Hq, Hk, Lk, Lq, d, tile, G, seed=11, pow2_v=True)
+    blk = np.arange(Lk) // tile
+    v16 = (c["v8"].astype(np.float64) * c["vs"][:, :, blk, None].astype(np.float64)).astype(np.float16)
+    assert np.array_equal(v16.astype(np.float64), c["v8"].astype(np.float64) * c["vs"][:, :, blk, None].astype(np.float64))
+    rows = [(b, h, c["off"] + i) for b in range(B) for h in range(Hq) for i in range(0, Lq, 7)] + \
+           [(b, h, Lk - 1) for b in range(B) for h in range(Hq)]
+    ref, ref_lse, _ = oracle.attention_rows(c["p"], c["q16"], c["k16"], np.ascontiguousarray(v16.view(np.uint16)),
+                                            c["q8"], c["k8"], c["qs"], c["ks"], c["words"], rows)
+    out, lse = _chunk_run(c)
+    for n, (b, h, i) in enumerate(rows):
+        assert np.abs(out[b, h, i - c["off"]] - ref[n]).max() < 1e-12
+        assert abs(lse[b, h, i - c["off"]] - ref_lse[n]) < 1e-12
+    assert c["route"].any() and not c["route"].all()
+
+
+def test_chunk_v8_of_one_query_is_the_decode_step():
+    """L_q = 1 with single-row query blocks: the chunk is the decode step over the same cache (the decode oracle
+    quantises the query row itself and takes one mask row per KV head)."""
+    B, Hq, Hk, Lk, d, tile, G = 2, 4, 2, 257, 32, 64, 1
+    c = _chunk_case(B, Hq, Hk, Lk, 1, d, tile, G, seed=12, blk_q=1)
+    out, lse = _chunk_run(c)
+    last = c["route"][:, :, c["p"].T_m - 1]                               # the mask row of the last query tile
+    ref, ref_lse = od.decode(np.ascontiguousarray(c["chunk"]["q16"][:, :, 0]), c["k16"], c["k8"], c["ks"], c["v8"],
+                             c["vs"], od.pack_row(last), np.full(B, Lk), tile, G)
+    assert np.abs(out[:, :, 0] - ref).max() < 1e-12 and np.abs(lse[:, :, 0] - ref_lse).max() < 1e-12
+    q8_row, dq_row = od.quantize_query(np.ascontiguousarray(c["chunk"]["q16"][:, :, 0]))
+    assert np.array_equal(q8_row, c["chunk"]["q8"][:, :, 0]) and np.array_equal(dq_row, c["chunk"]["qs"][:, :, 0])
+
+
+def test_chunk_v8_brute_force_loops():
+    B, Hq, Hk, Lk, Lq, d, tile, G = 1, 2, 1, 96, 32, 8, 32, 2
+    c = _chunk_case(B, Hq, Hk, Lk, Lq, d, tile, G, seed=13)
+    out, lse = _chunk_run(c)
+    half = lambda bits: float(np.array(bits, np.uint16).view(np.float16))
+    scale = 1.0 / math.sqrt(d)
+    for hq in range(Hq):
+        for i in (0, 5, 31):
+            cpos = c["off"] + i
+            s = []
+            for j in range(cpos + 1):
+                g = j // (tile * G)
+                if (int(c["words"][0, 0, cpos // tile, g >> 5]) >> (g & 31)) & 1:
+                    dot = sum(int(a) * int(b) for a, b in zip(c["chunk"]["q8"][0, hq, i], c["k8"][0, 0, j]))
+                    s.append(float(c["chunk"]["qs"][0, hq, i // tile]) * float(c["ks"][0, 0, j // tile]) * dot * scale)
+                else:
+                    s.append(sum(half(a) * half(b) for a, b in zip(c["chunk"]["q16"][0, hq, i], c["k16"][0, 0, j])) * scale)
+            m = max(s)
+            w = [math.exp(x - m) for x in s]
+            for e in range(d):
+                o = sum(w[j] * float(c["vs"][0, 0, j // tile]) * int(c["v8"][0, 0, j, e]) for j in range(cpos + 1)) / sum(w)
+                assert abs(o - out[0, hq, i, e]) < 1e-12
+            assert abs(m + math.log(sum(w)) - lse[0, hq, i]) < 1e-12
+    assert c["route"].any() and not c["route"].all()
