@@ -546,6 +546,20 @@ def main():
         fl = 4.0 * w.heads * w.head_dim * (float(Lq) * off + float(Lq) ** 2 / 2.0)
         line["chunk"] = {"chunk_len": Lq, "context_len": w.seqlen, "attention_ms": ms,
                          "tflops": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s"}
+        # the same chunk against an INT8 value cache (conversion kernel + fused kernel with delta_V folded into P)
+        _, v8f, _, vsf = tm.tilemix_quantize_qk(p, kd, vd)
+        work8 = torch.empty(tm.tilemix_chunk_v8_workspace_size(pc, w.seqlen), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            tm.tilemix_attention_fwd_chunk_v8(pc, w.seqlen, qc, kd, v8f, vsf, q8c, k8f, qsc, ksf, words_f, out=oc, workspace=work8)
+        c0.record(stream)
+        for _ in range(5):
+            tm.tilemix_attention_fwd_chunk_v8(pc, w.seqlen, qc, kd, v8f, vsf, q8c, k8f, qsc, ksf, words_f, out=oc, workspace=work8)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        ms8 = c0.elapsed_time(c1) / 5
+        line["chunk"]["int8_value_cache_ms"] = ms8
+        line["chunk"]["int8_value_cache_tflops"] = fl / (ms8 * 1e-3) / 1e12
+        del v8f, vsf, work8
     if world == 1 and not args.no_varlen and w.tile == 128 and w.head_dim == 128:
         # on-the-fly operand mode: no INT8 copies of Q and K and no scales in device memory; the kernel makes
         # them in shared memory (same mask, same result bit for bit -- checked here on the full workload)

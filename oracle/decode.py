@@ -11,7 +11,10 @@ sequence attends to the first cache_len[b] cached keys:
 
 with q8, delta_q the blockwise quantiser of App. C applied to the single query row (block = the rows
 that exist), h_k = h_q // (H_q / H_k), and bit g of the mask row of h_k routing the keys
-[g*G*tile_n, (g+1)*G*tile_n).  Nothing here is shared with the CUDA path.
+[g*G*tile_n, (g+1)*G*tile_n).  `chunk_v8` is the same cache read by the last L_q tokens of a context (chunked
+prefill: causal alignment, blockwise Q8 as in the prefill oracle).  Both functions are pinned by
+tests/test_oracle_decode_pins.py (a library attention routine, the prefill oracle, each other, plain loops).
+Nothing here is shared with the CUDA path.
 """
 from __future__ import annotations
 
