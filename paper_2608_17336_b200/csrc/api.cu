@@ -174,6 +174,9 @@ int tilemix_quantize_qk(const tilemix_problem_t* p, const void* q_f16, const voi
     if ((do_q && (!aligned16(q_f16) || !aligned16(q_i8))) || (do_k && (!aligned16(k_f16) || !aligned16(k_i8))))
         return TILEMIX_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (do_q && do_k)
+        return launch_quantize_pair(q_f16, g.qs, g.Hq, g.blk_q, q_i8, q_scale, k_f16, g.ks, g.Hk, g.blk_k, k_i8, k_scale,
+                                    g.B, g.L, g.d, s);
     if (do_q && (rc = launch_quantize(q_f16, g.qs, g.B, g.Hq, g.L, g.d, g.blk_q, q_i8, q_scale, s))) return rc;
     if (do_k && (rc = launch_quantize(k_f16, g.ks, g.B, g.Hk, g.L, g.d, g.blk_k, k_i8, k_scale, s))) return rc;
     return TILEMIX_OK;

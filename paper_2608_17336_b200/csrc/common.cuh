@@ -86,6 +86,9 @@ inline bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr
 int launch_quantize(const void* x, const int64_t stride[3], int B, int H, int L, int d, int blk,
                     int8_t* out, float* scale, cudaStream_t stream, const VarlenDev* vl = nullptr,
                     const int32_t* blk_off = nullptr, int total_blk = 0);
+int launch_quantize_pair(const void* q, const int64_t qstride[3], int Hq, int blk_q, int8_t* q8, float* qs,
+                         const void* k, const int64_t kstride[3], int Hk, int blk_k, int8_t* k8, float* ks,
+                         int B, int L, int d, cudaStream_t stream);
 int launch_pack(const Geometry& g, const uint8_t* route, uint32_t pack_flags, uint32_t* words,
                 unsigned long long* counts, cudaStream_t stream, const VarlenDev* vl = nullptr);
 int launch_attention(const Geometry& g, const void* q, const void* k, const void* v,
