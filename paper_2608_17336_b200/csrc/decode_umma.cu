@@ -638,8 +638,18 @@ int encode_cache_map(EncodeTiledFn enc, CUtensorMap* tm, const void* base, int e
 template <int R>
 int launch_r(const DecodeParams& prm, const CUtensorMap& tk8, const CUtensorMap& tk16, cudaStream_t stream) {
     auto kernel = prm.k16 != nullptr ? decode_umma_kernel<R, true> : decode_umma_kernel<R, false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    // the kernel's shared-memory attribute is set once per device and instance
+    constexpr int kMaxDev = 64;
+    static std::atomic<int> attr_set[kMaxDev][2];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return static_cast<int>(e);
+    const int which = prm.k16 != nullptr ? 1 : 0;
+    if (dev < 0 || dev >= kMaxDev || attr_set[dev][which].load(std::memory_order_acquire) == 0) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return static_cast<int>(e);
+        if (dev >= 0 && dev < kMaxDev) attr_set[dev][which].store(1, std::memory_order_release);
+    }
     const dim3 grid(prm.n_splits, prm.Hk, prm.B);
     // programmatic dependent launch: this grid's set-up overlaps the tail of the prepare kernel
     cudaLaunchConfig_t cfg = {};
@@ -656,11 +666,15 @@ int launch_r(const DecodeParams& prm, const CUtensorMap& tk8, const CUtensorMap&
 }  // namespace
 
 int launch_decode_umma(int R, const DecodeParams& prm, cudaStream_t stream) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
-    if (e != cudaSuccess) return static_cast<int>(e);
-    if (qres != cudaDriverEntryPointSuccess || sym == nullptr) return static_cast<int>(cudaErrorNotSupported);
+    static std::atomic<void*> encoder{nullptr};      // the driver's tensor-map encoder, looked up once
+    void* sym = encoder.load(std::memory_order_acquire);
+    if (sym == nullptr) {
+        cudaDriverEntryPointQueryResult qres;
+        const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return static_cast<int>(e);
+        if (qres != cudaDriverEntryPointSuccess || sym == nullptr) return static_cast<int>(cudaErrorNotSupported);
+        encoder.store(sym, std::memory_order_release);
+    }
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(sym);
     CUtensorMap tk8, tk16;
     int rc = encode_cache_map(enc, &tk8, prm.k8, 1, prm, 128);

@@ -249,13 +249,21 @@ bool stream_eligible(const int64_t stride[3], int d, int blk) {
 int launch_stream(QuantJobs& jobs, cudaStream_t stream) {
     if (jobs.total > 0x3fffffff) return cudaErrorInvalidConfiguration;
     jobs.wait_limit_ns = g_wait_limit_ns.load();
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return static_cast<int>(e);
+    // SM count and the kernel's shared-memory attribute: asked for / set once per device
+    constexpr int kMaxDev = 64;
+    static std::atomic<int> sm_count[kMaxDev];
     constexpr int kSmem = kStreamStages * kStageBytes;
-    e = cudaFuncSetAttribute(quantize_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return static_cast<int>(e);
+    int sms = (dev >= 0 && dev < kMaxDev) ? sm_count[dev].load(std::memory_order_acquire) : 0;
+    if (sms == 0) {
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(quantize_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (e != cudaSuccess) return static_cast<int>(e);
+        if (dev >= 0 && dev < kMaxDev) sm_count[dev].store(sms, std::memory_order_release);
+    }
     const int grid = jobs.total < sms ? jobs.total : sms;
     quantize_stream_kernel<<<grid, kStreamThreads, kSmem, stream>>>(jobs);
     g_launch_count.fetch_add(1);
