@@ -137,12 +137,77 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     // where it is about to write that record.
     const int len = min(max(prm.cache_len_raw[b], 0), prm.max_len);
     const int n_tiles = (len + T - 1) / T;
-    const int per_split = (n_tiles + prm.n_splits - 1) / prm.n_splits;
-    const int t0 = split * per_split, t1 = min(n_tiles, t0 + per_split);
+    const uint32_t* wrow = prm.words != nullptr
+        ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : b) * prm.Hk + hk) * prm.W : nullptr;
+    // The splits of a row share its BYTES, not its tiles: a routing group costs 2 units per tile on the INT8 route
+    // (K8 + V8) and 3 on the FP16 route, and with one wave of CTAs the one with the most bytes ends last.  Split
+    // k takes the groups [bound(k C / n), bound((k + 1) C / n)), C the cost of the row and bound(x) the first
+    // group at which the running cost reaches x; every thread computes the two bounds it needs (a scan over at
+    // most W mask words).
+    const int n_groups = (n_tiles + prm.G - 1) / prm.G;
+    auto word_bits = [&](int w) -> int { return min(32, n_groups - 32 * w); };                  // groups of word w that exist
+    auto word_cost = [&](int w, int nb) -> int {                                                  // cost of its first nb groups
+        const uint32_t bits = wrow != nullptr ? wrow[w] & (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u)) : 0u;
+        return 3 * nb - __popc(bits);
+    };
+    int total = 0;
+    for (int w = 0; 32 * w < n_groups; ++w) total += word_cost(w, word_bits(w));
+    auto bound = [&](long long x) -> int {
+        if (x <= 0) return 0;
+        int acc = 0, w = 0;
+        for (; 32 * w < n_groups; ++w) {
+            const int c = word_cost(w, word_bits(w));
+            if (acc + c >= x) break;
+            acc += c;
+        }
+        if (32 * w >= n_groups) return n_groups;
+        const int nb = word_bits(w);
+        int i = 1;
+        while (i < nb && acc + word_cost(w, i) < x) ++i;    // smallest i with the cost of i groups of this word >= x - acc
+        return 32 * w + i;
+    };
+    const int g0 = bound(static_cast<long long>(split) * total / prm.n_splits);
+    const int g1 = split + 1 == prm.n_splits ? n_groups : bound(static_cast<long long>(split + 1) * total / prm.n_splits);
+    const int t0 = min(n_tiles, g0 * prm.G), t1 = min(n_tiles, g1 * prm.G);
     const int n_it = t1 - t0;
     const int n_pairs = (n_it + 1) / 2;   // the softmax warps take two key tiles per step
     const int n_parts = kStreams * prm.n_splits;   // partial results per query head in the workspace
     const int64_t out_row0 = (static_cast<int64_t>(b) * prm.Hq + hk * R) * n_parts + kStreams * split;   // + r * n_parts + stream
+
+    // Query row r of this KV head: FP16 copy and blockwise INT8 (block = the row), both as K-major operand rows in
+    // shared memory (to_smem), and -- from the one split of the row that starts at its first group -- the quantised
+    // row and its scale to the caller's buffers.
+    const bool q_writer = g0 == 0 && (g1 > 0 || split + 1 == prm.n_splits);
+    auto prep_query_row = [&](int r, bool to_smem) {
+        const int hq = hk * R + r;
+        const __half* qrow = prm.q + (static_cast<int64_t>(b) * prm.Hq + hq) * D;
+        float v[D / 32];
+        float amax = 0.f;
+#pragma unroll
+        for (int x = 0; x < D / 32; ++x) {
+            v[x] = __half2float(qrow[lane + 32 * x]);
+            amax = fmaxf(amax, fabsf(v[x]));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        const float delta = __fdiv_rn(amax, 127.f);
+#pragma unroll
+        for (int x = 0; x < D / 32; ++x) {
+            const int e = lane + 32 * x;
+            int q8 = 0;
+            if (amax > 0.f) q8 = max(-127, min(127, __float2int_rn(__fdiv_rn(v[x], delta))));
+            if (to_smem) {
+                *reinterpret_cast<__half*>(sm + kOffQ16 + (e >> 6) * 1024 + r * 128 + ((((e & 63) >> 3) ^ r) << 4) + (e & 7) * 2) = qrow[e];
+                *reinterpret_cast<int8_t*>(sm + kOffQ8 + r * 128 + (((e >> 4) ^ r) << 4) + (e & 15)) = static_cast<int8_t>(q8);
+            }
+            if (q_writer && prm.q8_out != nullptr)
+                prm.q8_out[(static_cast<int64_t>(b) * prm.Hq + hq) * D + e] = static_cast<int8_t>(q8);
+        }
+        if (lane == 0) {
+            if (to_smem) sh.dq[r] = delta;
+            if (q_writer && prm.qs_out != nullptr) prm.qs_out[static_cast<int64_t>(b) * prm.Hq + hq] = delta;
+        }
+    };
 
     if (n_it <= 0) {                      // a split without keys: the merge skips it
         for (int idx = tid; idx < kStreams * R * D; idx += kThreads) {
@@ -153,14 +218,13 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             prm.m_part[out_row0 + static_cast<int64_t>(tid % R) * n_parts + tid / R] = -INFINITY;
             prm.z_part[out_row0 + static_cast<int64_t>(tid % R) * n_parts + tid / R] = 0.f;
         }
+        if (q_writer && warp < R) prep_query_row(warp, false);   // (a row without keys still reports its quantised query)
         leave();
         return;
     }
 
     const float* dk = prm.k_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.n_blk;
     const float* dv = prm.v_scale + (static_cast<int64_t>(b) * prm.Hk + hk) * prm.n_blk;
-    const uint32_t* wrow = prm.words != nullptr
-        ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : b) * prm.Hk + hk) * prm.W : nullptr;
     auto route_of = [&](int tile) -> bool {
         if (wrow == nullptr) return false;
         const int grp = tile / prm.G;
@@ -272,36 +336,7 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
             meta[i] = make_float2(route_of(tile) ? dk[tile] : -1.f, dv[tile]);
         }
         ptx::bar_sync_named(1, kThreads - 32);
-        if (warp >= kConvWarp0 && warp < kConvWarp0 + R) {
-            // query row r of this KV head: FP16 copy and blockwise INT8 (block = the row), both as K-major operand rows
-            const int r = warp - kConvWarp0;
-            const int hq = hk * R + r;
-            const __half* qrow = prm.q + (static_cast<int64_t>(b) * prm.Hq + hq) * D;
-            float v[D / 32];
-            float amax = 0.f;
-    #pragma unroll
-            for (int x = 0; x < D / 32; ++x) {
-                v[x] = __half2float(qrow[lane + 32 * x]);
-                amax = fmaxf(amax, fabsf(v[x]));
-            }
-    #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            const float delta = __fdiv_rn(amax, 127.f);
-    #pragma unroll
-            for (int x = 0; x < D / 32; ++x) {
-                const int e = lane + 32 * x;
-                int q8 = 0;
-                if (amax > 0.f) q8 = max(-127, min(127, __float2int_rn(__fdiv_rn(v[x], delta))));
-                *reinterpret_cast<__half*>(sm + kOffQ16 + (e >> 6) * 1024 + r * 128 + ((((e & 63) >> 3) ^ r) << 4) + (e & 7) * 2) = qrow[e];
-                *reinterpret_cast<int8_t*>(sm + kOffQ8 + r * 128 + (((e >> 4) ^ r) << 4) + (e & 15)) = static_cast<int8_t>(q8);
-                if (split == 0 && prm.q8_out != nullptr)
-                    prm.q8_out[(static_cast<int64_t>(b) * prm.Hq + hq) * D + e] = static_cast<int8_t>(q8);
-            }
-            if (lane == 0) {
-                sh.dq[r] = delta;
-                if (split == 0 && prm.qs_out != nullptr) prm.qs_out[static_cast<int64_t>(b) * prm.Hq + hq] = delta;
-            }
-        }
+        if (warp >= kConvWarp0 && warp < kConvWarp0 + R) prep_query_row(warp - kConvWarp0, true);
         ptx::fence_proxy_async_smem();        // operand tiles written with ordinary stores, read by the tensor pipe
         ptx::bar_sync_named(1, kThreads - 32);
 

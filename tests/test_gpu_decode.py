@@ -196,3 +196,11 @@ def test_decode_more_tiles_per_split_than_the_staged_metadata():
     takes the rest from global memory; more than 32 routing groups per row, so more than one mask word."""
     q, k, v, route, lens = _case(1, 4, 1, 34000, 128, 128, 3, seed=52, lens=[33990], f8=0.5)
     _check(q, k, v, route, lens, 128, 3, n_splits=1)
+
+
+def test_decode_zero_length_and_one_key_rows_on_the_tcgen05_form():
+    """head_dim 128 with 128-key tiles: a sequence without keys (zero output, lse = -inf, its quantised query still
+    reported), one with a single key, and splits that get no group at all (more splits than groups)."""
+    q, k, v, route, lens = _case(4, 4, 2, 300, 128, 128, 1, seed=53, lens=[300, 0, 1, 128])
+    _check(q, k, v, route, lens, 128, 1)
+    _check(q, k, v, route, lens, 128, 1, n_splits=5)
