@@ -42,6 +42,25 @@ def test_quantize_bit_exact(B, Hh, L, d, blk):
         assert (xs.cpu().numpy().view(np.uint32) == rs.view(np.uint32)).all()
 
 
+@pytest.mark.parametrize("B,Hq,Hk,L,d,blk_q,blk_k", [(2, 8, 2, 3000, 128, 128, 64), (1, 4, 1, 20000, 128, 128, 128),
+                                                     (3, 2, 1, 130, 64, 64, 64)])
+def test_quantize_pair_of_different_shapes_in_one_launch(B, Hq, Hk, L, d, blk_q, blk_k):
+    """Q and K with different head counts and block sizes (grouped-query attention, the paper's BLK_K = BLOCK_N / 2)
+    go through one launch of the streaming quantiser; more blocks than the persistent CTAs take in one round; a
+    ragged last block; values on rounding ties (multiples of 1/2 scaled so that x / delta hits .5)."""
+    b = _binding()
+    gen = torch.Generator().manual_seed(L + Hq)
+    q = (torch.randint(-254, 255, (B, Hq, L, d), generator=gen).float() * 0.5).half()      # max |x| = 127 -> delta = 1: ties
+    q[:, :, 0, 0] = 127.0
+    k = (torch.randn((B, Hk, L, d), generator=gen) * 2).half()
+    p = b.problem(B, Hq, Hk, L, d, max(blk_q, blk_k), max(blk_q, blk_k), quant_blk_q=blk_q, quant_blk_k=blk_k)
+    q8, k8, qs, ks = b.tilemix_quantize_qk(p, q.cuda(), k.cuda())
+    for x, x8, xs, blk in ((q, q8, qs, blk_q), (k, k8, ks, blk_k)):
+        r8, rs = oracle.quantize(H.np_bits(x), blk)
+        assert (x8.cpu().numpy() == r8).all()
+        assert (xs.cpu().numpy().view(np.uint32) == rs.view(np.uint32)).all()
+
+
 def test_quantize_strided_input():
     b = _binding()
     B, Hh, L, d = 2, 3, 384, 128
