@@ -1,10 +1,11 @@
 // Decode step over an INT8 key/value cache (App. C, "Additional Execution Interfaces"): one query
 // token per sequence, keys split over CTAs, the H_q/H_k query heads of a KV head served together.
 // HBM-bound: a cached token costs d bytes of K8 (or 2d of FP16 K on the FP16 route) plus d bytes of
-// V8, each read once: the tiles are contiguous in the cache and are streamed into a shared-memory ring
-// by untiled bulk copies, a tile ahead of their use.  The H_q/H_k query rows of a KV head are the rows of
-// a 16-row warp-level tensor-core operand (the 64-row minimum of tcgen05 has no use for 1..8 rows); on
-// the CUDA cores alone the step is instruction-bound at about a third of the HBM rate.
+// V8, each read once.  This file holds the host entry points, the preparation and merge kernels, and the
+// warp-level form of the step for head_dim 64 or 64-key tiles: the tiles are streamed into a shared-memory
+// ring by untiled bulk copies, a tile ahead of their use, and the H_q/H_k query rows of a KV head are the
+// rows of a 16-row warp-level tensor-core operand.  head_dim 128 with 128-key tiles runs the tcgen05 form
+// (decode_umma.cu), where the KEYS are the MMA rows.
 #include <cuda_fp16.h>
 #include <math.h>
 
