@@ -204,3 +204,12 @@ def test_decode_zero_length_and_one_key_rows_on_the_tcgen05_form():
     q, k, v, route, lens = _case(4, 4, 2, 300, 128, 128, 1, seed=53, lens=[300, 0, 1, 128])
     _check(q, k, v, route, lens, 128, 1)
     _check(q, k, v, route, lens, 128, 1, n_splits=5)
+
+
+@pytest.mark.parametrize("rep", [1, 2, 4, 8])
+def test_decode_gqa_group_sizes_on_the_tcgen05_form(rep):
+    """head_dim 128 with 128-key tiles, H_q / H_k = 1, 2, 4, 8, a ragged cache of nine tiles and a mixed mask, with
+    one split per row (both softmax streams of a CTA get several steps) and with the library's choice."""
+    q, k, v, route, lens = _case(2, 2 * rep, 2, 1152, 128, 128, 1, seed=70 + rep, lens=[1100, 1152])
+    _check(q, k, v, route, lens, 128, 1, n_splits=1)
+    _check(q, k, v, route, lens, 128, 1)
