@@ -364,6 +364,8 @@ int tilemix_tensor_peak_probe(int int8, int n_mma, int* n_ctas, void* workspace,
  *   which = 1  the attention kernel's producer leaves out the copies of operand bundle 1 (V of key tile 0 and K of key
  *              tile 1) of every CTA, so an MMA issuer's wait for that bundle runs out after wait_limit_ns
  *   which = 2  the decode step's producer leaves out the second tile of every split
+ *   which = 3  the streaming quantiser's producer leaves out the second block of every CTA; the quantiser has no
+ *              status record: a CTA that gives up writes NaN into the scales of the blocks it did not finish
  *   which = 0  normal operation, limit back to the default of 2 s (wait_limit_ns is ignored)
  * Returns TILEMIX_OK or TILEMIX_ERR_SHAPE. */
 int tilemix_test_drop_copy(int which, uint64_t wait_limit_ns);

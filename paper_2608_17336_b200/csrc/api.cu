@@ -456,7 +456,7 @@ const char* tilemix_status_string(int code) {
 uint64_t tilemix_launch_count(void) { return g_launch_count.load(); }
 
 int tilemix_test_drop_copy(int which, uint64_t wait_limit_ns) {
-    if (which < 0 || which > 2) return TILEMIX_ERR_SHAPE;
+    if (which < 0 || which > 3) return TILEMIX_ERR_SHAPE;
     g_test_drop.store(which);
     g_wait_limit_ns.store(which == 0 || wait_limit_ns == 0 ? kDefaultWaitLimitNs : wait_limit_ns);
     return TILEMIX_OK;

@@ -16,7 +16,7 @@ extern std::atomic<uint64_t> g_launch_count;
 
 // Testing aid (tilemix_test_drop_copy): which producer leaves out one copy, and the limit of the bounded waits.
 constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
-extern std::atomic<int> g_test_drop;                 // 0 none, 1 attention kernel, 2 decode step
+extern std::atomic<int> g_test_drop;                 // 0 none, 1 attention kernel, 2 decode step, 3 streaming quantiser
 extern std::atomic<uint64_t> g_wait_limit_ns;
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

@@ -122,6 +122,7 @@ struct QuantJobs {
     QuantJob j[2];
     int n_jobs, total, d;
     unsigned long long wait_limit_ns;
+    int test_drop_block;       // testing aid: the producer leaves out the copy of this block of every CTA (-1: none)
 };
 
 __global__ void __launch_bounds__(kStreamThreads, 1) quantize_stream_kernel(const QuantJobs jobs) {
@@ -179,6 +180,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) quantize_stream_kernel(cons
             for (int t = 0; t < n_mine; ++t) {
                 const int s = t % kStreamStages;
                 if (t >= kStreamStages && !wait(&empty[s], ((t / kStreamStages) - 1) & 1)) break;
+                if (t == jobs.test_drop_block) continue;   // testing aid: this block never lands, the consumers' wait runs out
                 const Where w = locate(t);
                 const uint32_t bytes = static_cast<uint32_t>(w.rows) * d * 2u;
                 const uint32_t bar = ptx::smem_u32(&full[s]);
@@ -233,9 +235,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) quantize_stream_kernel(cons
         // A wait ran out (a copy that never landed): the copies still in flight land before the shared memory is
         // given back, and the scales of the blocks that were not finished are marked with NaN.
         if (warp == kStreamGroups * kStreamWarps && lane == 0) {
-            for (int t = max(0, issued - kStreamStages); t < issued; ++t)
+            for (int t = max(0, issued - kStreamStages); t < issued; ++t) {
+                if (t == jobs.test_drop_block) continue;
                 for (int spin = 0; spin < (1 << 16); ++spin)
                     if (ptx::mbar_try_wait(ptx::smem_u32(&full[t % kStreamStages]), (t / kStreamStages) & 1)) break;
+            }
         }
         if (warp < kStreamGroups * kStreamWarps && (tid % (kStreamWarps * 32)) == 0)
             for (int t = max(done, warp / kStreamWarps); t < n_mine; t += kStreamGroups) *locate(t).scale = __int_as_float(0x7fc00000);
@@ -249,6 +253,7 @@ bool stream_eligible(const int64_t stride[3], int d, int blk) {
 int launch_stream(QuantJobs& jobs, cudaStream_t stream) {
     if (jobs.total > 0x3fffffff) return cudaErrorInvalidConfiguration;
     jobs.wait_limit_ns = g_wait_limit_ns.load();
+    jobs.test_drop_block = g_test_drop.load() == 3 ? 1 : -1;
     // SM count and the kernel's shared-memory attribute: asked for / set once per device
     constexpr int kMaxDev = 64;
     static std::atomic<int> sm_count[kMaxDev];

@@ -79,3 +79,30 @@ def test_decode_wait_runs_out_and_the_kernel_returns(drop):
     again = tm.tilemix_decode_int8kv(p, q, k, k8, ks, v8, vs, words, lens, workspace=good["workspace"])
     assert tm.tilemix_read_status(again["workspace"])[0] == 0
     assert torch.equal(again["out"], good["out"])
+
+
+def test_quantiser_wait_runs_out_and_the_kernel_returns(drop):
+    """The streaming quantiser has no status record: a CTA whose wait for a block runs out stops, waits for its copies
+    in flight and marks the scales of the blocks it did not finish with NaN."""
+    from paper_2608_17336_b200 import binding as tm
+    B, Hh, L, d = 1, 32, 4096, 128                     # 2 x 1024 blocks: every persistent CTA has well over two
+    gen = torch.Generator(device="cpu").manual_seed(93)
+    q = torch.randn((B, Hh, L, d), generator=gen).half().to(DEV)
+    k = torch.randn((B, Hh, L, d), generator=gen).half().to(DEV)
+    p = tm.problem(B, Hh, Hh, L, d, 128, 128)
+    good = tm.tilemix_quantize_qk(p, q, k)
+    assert all(torch.isfinite(x).all() for x in good[2:])
+    drop(3, 2_000_000)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    bad = tm.tilemix_quantize_qk(p, q, k)
+    t1.record()
+    torch.cuda.synchronize()
+    scales = torch.cat([bad[2].flatten(), bad[3].flatten()])          # the launch's blocks in order: Q's, then K's
+    n_ctas = torch.cuda.get_device_properties(0).multi_processor_count
+    assert torch.isnan(scales[n_ctas:2 * n_ctas]).all()               # block 1 of CTA c is block c + n_ctas of the launch
+    assert torch.isfinite(scales[:n_ctas]).all()                      # block 0 of every CTA was finished
+    assert t0.elapsed_time(t1) < 500.0
+    drop(0)
+    again = tm.tilemix_quantize_qk(p, q, k)
+    assert all(torch.equal(a, g) for a, g in zip(again, good))
