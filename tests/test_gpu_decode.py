@@ -213,3 +213,41 @@ def test_decode_gqa_group_sizes_on_the_tcgen05_form(rep):
     q, k, v, route, lens = _case(2, 2 * rep, 2, 1152, 128, 128, 1, seed=70 + rep, lens=[1100, 1152])
     _check(q, k, v, route, lens, 128, 1, n_splits=1)
     _check(q, k, v, route, lens, 128, 1)
+
+
+def test_decode_at_the_bench_workload_size():
+    """8 sequences x 32768 cached tokens, H_q 32 / H_k 8, d 128, G = 4, 75 % INT8 groups, ragged lengths in the last
+    two sequences -- the shapes and the launch configuration (library-chosen splits) that bench.py times.  Every output
+    of three of the eight sequences against the oracle, after the cache the oracle is given was checked."""
+    from paper_2608_17336_b200 import binding as tm
+    B, Hq, Hk, L, d, tile, G = 8, 32, 8, 32768, 128, 128, 4
+    gen = torch.Generator(device="cpu").manual_seed(81)
+    q = torch.randn((B, Hq, d), generator=gen).half()
+    k = torch.randn((B, Hk, L, d), generator=gen).half()
+    v = torch.randn((B, Hk, L, d), generator=gen).half()
+    rng = np.random.default_rng(82)
+    route = (rng.random((1, Hk, -(-L // (tile * G)))) < 0.75).astype(np.uint8)
+    lens = np.asarray([L, L, L, L, L, L, 30001, 17], np.int32)
+    dev = torch.device("cuda:0")
+    kd, vd = k.to(dev), v.to(dev)
+    k8, v8, ks, vs = tm.tilemix_quantize_qk(tm.problem(B, Hk, Hk, L, d, tile, tile), kd, vd)
+    p = tm.decode_problem(B, Hq, Hk, d, L, tile, G)
+    words = torch.from_numpy(od.pack_row(route).view(np.int32)).to(dev)
+    res = tm.tilemix_decode_int8kv(p, q.to(dev), kd, k8, ks, v8, vs, words, torch.from_numpy(lens).to(dev), want_lse=True)
+    torch.cuda.synchronize()
+    assert tm.tilemix_read_status(res["workspace"])[0] == 0
+    out = res["out"].float().cpu().numpy().astype(np.float64)
+    lse = res["lse"].cpu().numpy().astype(np.float64)
+    bits = lambda t: np.ascontiguousarray(t.view(torch.int16).numpy()).view(np.uint16)
+    for b in (0, 6, 7):
+        sl = slice(b, b + 1)
+        k16, v16 = bits(k[sl]), bits(v[sl])
+        k8_ref, ks_ref = oracle.quantize(k16, tile)
+        v8_ref, vs_ref = oracle.quantize(v16, tile)
+        assert np.array_equal(k8[sl].cpu().numpy(), k8_ref) and np.array_equal(v8[sl].cpu().numpy(), v8_ref)
+        assert np.array_equal(ks[sl].cpu().numpy().view(np.uint32), ks_ref.view(np.uint32))
+        assert np.array_equal(vs[sl].cpu().numpy().view(np.uint32), vs_ref.view(np.uint32))
+        ref, ref_lse = od.decode(bits(q[sl]), k16, k8_ref, ks_ref, v8_ref, vs_ref, od.pack_row(route), lens[sl], tile, G)
+        err = np.abs(out[sl] - ref)
+        assert (err <= ATOL * np.maximum(1.0, np.abs(ref))).all(), f"sequence {b}: max err {err.max():.3e}"
+        assert np.abs(lse[sl] - ref_lse).max() < 2e-3
