@@ -199,6 +199,11 @@ def test_decode_host_side_validation(lib):
     splits = (size - 512) // (8 * 32 * (128 * 4 + 8))
     assert splits >= 1 and size == 512 + 8 * 32 * splits * (128 * 4 + 8)
     assert b.tilemix_decode_workspace_size(b.decode_problem(1, 4, 1, 64, 64, 64, n_splits=7)) == 256 + 256 + 1024 + 2 * 256
+    # head_dim 128 with 128-key tiles (the tcgen05 form): one wave of CTAs by default (148 SMs / 64 rows = 2 splits),
+    # two partial results per split
+    assert splits == 2 * 2
+    three = b.tilemix_decode_workspace_size(b.decode_problem(8, 32, 8, 128, 32768, 128, 4, n_splits=3))
+    assert three == 512 + 8 * 32 * (2 * 3) * (128 * 4 + 8)
     for bad in (b.decode_problem(0, 32, 8, 128, 1024, 128), b.decode_problem(1, 6, 4, 128, 1024, 128),
                 b.decode_problem(1, 4, 4, 128, 0, 128), b.decode_problem(2, 4, 4, 128, 1024, 128, mask_batch=3)):
         assert lib.tilemix_decode_workspace_size(ctypes.byref(bad)) == 0
