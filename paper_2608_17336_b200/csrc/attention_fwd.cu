@@ -785,6 +785,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 // P = 2^(a*raw - m) is rounded to FP16, one pair per register.
                 const bool diag = (j == k_t);
                 bool redo = diag || u == 0 || prm.dbg_n > 0;
+                bool stored = false;      // P of the one-pass form has been sent to tensor memory
                 float alpha[2] = {1.f, 1.f}, sum[2] = {0.f, 0.f};
                 bool grow = false;
                 uint32_t p[2 * NB];
@@ -801,6 +802,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         const float addend[2] = {-m_run[0], -m_run[1]};
                         softmax_step_fast<NB, kInt8Exact, VS>(s, a, addend, p, sum, dv);
                     }
+                    // The store of P goes out before the vote, so that the vote's latency hides behind it; a rejected
+                    // step stores again below, after this store has been waited for.
+                    if constexpr (NB == 8) ptx::tmem_st16x128_x8(t_sh, p);
+                    else ptx::tmem_st16x128_x4(t_sh, p);
+                    stored = true;
                     redo = __any_sync(0xffffffffu, !(sum[0] <= exp2f(kAccept) && sum[1] <= exp2f(kAccept)));   // also true for a NaN
                 }
                 if (redo) {
@@ -895,8 +901,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                         ptx::tmem_st16x256_x4(t_o + c * 32, o);
                     }
                 }
-                if constexpr (NB == 8) ptx::tmem_st16x128_x8(t_sh, p);
-                else ptx::tmem_st16x128_x4(t_sh, p);
+                if (redo) {
+                    if (stored) ptx::tmem_wait_st();      // (the rejected one-pass store, before the same columns are stored again)
+                    if constexpr (NB == 8) ptx::tmem_st16x128_x8(t_sh, p);
+                    else ptx::tmem_st16x128_x4(t_sh, p);
+                }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 ptx::mbar_arrive(bar_p(t, h));
