@@ -302,7 +302,12 @@ typedef struct tilemix_decode {
     int32_t max_len;       /* token capacity of the caches (their token stride)             */
     int32_t tile_n, group; /* key tile = scale block; G key tiles per routing bit           */
     int32_t mask_batch;    /* 1 = one mask row per KV head shared by the batch, or == batch */
-    int32_t n_splits;      /* CTAs per (b, h_k); 0 = chosen by the library                  */
+    int32_t n_splits;      /* CTAs per (b, h_k); 0 = chosen by the library, the same for every (b, h_k);
+                            * -1 = chosen by the kernel per (b, h_k), for batches of unequal cache lengths: in
+                            * the tcgen05 form with batch * heads_kv <= 148 the CTAs of one wave are shared out
+                            * so that the largest number of cache bytes a CTA reads is as small as it can be
+                            * (a row gets clamp(ceil(bytes / tau), 1, cap) CTAs for the smallest tau that fits
+                            * the wave); elsewhere -1 means 0 */
     float softmax_scale;   /* <= 0 means 1/sqrt(head_dim)                                   */
 } tilemix_decode_t;
 

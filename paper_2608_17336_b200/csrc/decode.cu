@@ -425,7 +425,10 @@ decode_kernel(const DecodeParams prm) {
     }
 }
 
-// Merge of the splits: m = max m_s, z = sum z_s 2^(m_s - m), O = sum O~_s 2^(m_s - m) / z.
+// Merge of the splits: m = max m_s, z = sum z_s 2^(m_s - m), O = sum O~_s 2^(m_s - m) / z.  One block per query head,
+// one thread per output element.  The parts are taken 32 at a time: lane s of every warp loads (m_s, z_s) and the
+// weights are shared by shuffles, so that the loads of O~_s depend on one round trip only and are in flight
+// together (a part that nobody wrote has m_s = -inf, weight 0, and is not loaded).
 template <int D>
 __global__ void __launch_bounds__(D)
 decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ m_part,
@@ -433,17 +436,28 @@ decode_merge_kernel(const float* __restrict__ o_part, const float* __restrict__ 
                     float* __restrict__ lse) {
     ptx::griddep_wait();   // (when launched as a programmatic dependent of the step kernel)
     const int64_t row = blockIdx.x;
-    const int e = threadIdx.x;
-    float m = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) m = fmaxf(m, m_part[row * n_splits + s]);
-    float z = 0.f, o = 0.f;
-    if (m > -INFINITY) {
-        for (int s = 0; s < n_splits; ++s) {
-            const float ms = m_part[row * n_splits + s];
-            if (ms == -INFINITY) continue;
-            const float w = exp2f(ms - m);
-            z += z_part[row * n_splits + s] * w;
-            o += o_part[(row * n_splits + s) * D + e] * w;
+    const int e = threadIdx.x, lane = e & 31;
+    float m = -INFINITY, z = 0.f, o = 0.f;
+    for (int s0 = 0; s0 < n_splits; s0 += 32) {
+        const int s = s0 + lane;
+        const float ms = s < n_splits ? m_part[row * n_splits + s] : -INFINITY;
+        const float zs = s < n_splits ? z_part[row * n_splits + s] : 0.f;
+        float mc = ms;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) mc = fmaxf(mc, __shfl_xor_sync(0xffffffffu, mc, d));
+        const float m_new = fmaxf(m, mc);
+        if (m_new == -INFINITY) continue;                    // (the same in every lane)
+        const float back = m == -INFINITY ? 0.f : exp2f(m - m_new);
+        const float w = ms == -INFINITY ? 0.f : exp2f(ms - m_new);
+        const float zw = ms == -INFINITY ? 0.f : zs * w;
+        z *= back; o *= back; m = m_new;
+        const int cnt = min(32, n_splits - s0);
+        const float* src = o_part + (row * n_splits + s0) * D + e;
+#pragma unroll 8
+        for (int i = 0; i < cnt; ++i) {
+            const float wi = __shfl_sync(0xffffffffu, w, i);
+            z += __shfl_sync(0xffffffffu, zw, i);
+            if (wi != 0.f) o += src[static_cast<int64_t>(i) * D] * wi;
         }
     }
     out[row * D + e] = __float2half_rn(z > 0.f ? o / z : 0.f);
@@ -480,6 +494,8 @@ int launch_r(int R, const DecodeParams& prm, __half* out, float* lse, cudaStream
 }
 
 constexpr size_t kDecodeStatusBytes = 256;   // status record of the bounded waits
+constexpr int kDecodeWave = 148;             // CTAs of one wave of the tcgen05 form (one per SM)
+constexpr int kDecodeBalanceRows = 160;      // rows of a batch whose splits that kernel can balance
 
 // Before the step: clears the status record and copies the cache lengths, clamped to [0, max_len], into the
 // workspace (they live on the device, so the host cannot check them; the step itself reads the copy).
@@ -496,13 +512,14 @@ size_t decode_len_bytes(int B) { return (static_cast<size_t>(B) * sizeof(int32_t
 struct DecodeGeometry {
     int n_blk, T_mask, W, n_splits;
     int n_parts;            // partial results per query head in the workspace (the tcgen05 form writes two per split)
+    int balanced, n_ctas, split_cap;   // tcgen05 form with an automatic split count: see DecodeParams
     size_t o_bytes, mz_bytes;
 };
 
 int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     if (p == nullptr) return TILEMIX_ERR_NULL;
     if (p->batch <= 0 || p->heads_q <= 0 || p->heads_kv <= 0 || p->head_dim <= 0 || p->max_len <= 0 ||
-        p->tile_n <= 0 || p->group <= 0 || p->n_splits < 0)
+        p->tile_n <= 0 || p->group <= 0 || p->n_splits < -1)
         return TILEMIX_ERR_SHAPE;
     if (p->heads_q % p->heads_kv != 0) return TILEMIX_ERR_SHAPE;
     if (p->mask_batch != 1 && p->mask_batch != p->batch) return TILEMIX_ERR_SHAPE;
@@ -513,17 +530,32 @@ int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     g->n_blk = static_cast<int>(ceil_div(p->max_len, p->tile_n));
     g->T_mask = static_cast<int>(ceil_div(p->max_len, static_cast<int64_t>(p->group) * p->tile_n));
     g->W = static_cast<int>(ceil_div(g->T_mask, 32));
-    int splits = p->n_splits;
+    // n_splits: > 0 as given, 0 chosen here (the same for every row), -1 chosen here and, where the kernel can do
+    // it, shared out over the rows by the kernel
+    const bool balance = p->n_splits == -1;
+    int splits = balance ? 0 : p->n_splits;
     const bool umma = p->head_dim == 128 && p->tile_n == 128;   // the tcgen05 form of the step (decode_umma.cu)
+    g->balanced = 0; g->n_ctas = 0; g->split_cap = 0;
     if (splits == 0) {
         if (umma) {
             // one CTA per SM, HBM-bound once every SM streams: a single wave, as many splits as fit into it
             // (measured at 8 x 8 KV heads and 32K keys: 2 splits = 128 CTAs 104 us, 9 splits = 3.9 waves 123 us),
             // at least four key tiles per split
-            const int64_t want = 148 / (static_cast<int64_t>(p->batch) * p->heads_kv);
+            const int64_t n_rows = static_cast<int64_t>(p->batch) * p->heads_kv;
+            const int64_t want = kDecodeWave / n_rows;
             splits = static_cast<int>(want < 1 ? 1 : want);
             const int cap = g->n_blk / 4 > 0 ? g->n_blk / 4 : 1;
             if (splits > cap) splits = cap;
+            // On request, for a batch whose rows fit one wave: the kernel shares the wave's CTAs out by the rows'
+            // cost (cache length, FP16-routed groups), up to split_cap to a row; the workspace has room for that
+            // many.  Not the default: with rows of one length it gains ~3 % (the FP16-routed groups differ) and
+            // loses ~5 us -- a full wave leaves no SM on which the merge kernel can wait ahead of time.
+            if (balance && n_rows <= kDecodeWave && n_rows <= kDecodeBalanceRows) {
+                int row_cap = 8 * splits < 16 ? 16 : 8 * splits;
+                if (row_cap > cap) row_cap = cap;
+                const int64_t ctas = n_rows * row_cap < kDecodeWave ? n_rows * row_cap : kDecodeWave;
+                g->balanced = 1; g->n_ctas = static_cast<int>(ctas); g->split_cap = row_cap;
+            }
         } else {
             // at most two full waves of two CTAs per SM over the whole batch (measured: more splits cost
             // more in per-CTA set-up and merge than they gain, and a third, partial wave idles a quarter
@@ -537,7 +569,7 @@ int resolve_decode(const tilemix_decode_t* p, DecodeGeometry* g) {
     if (splits > g->n_blk) splits = g->n_blk;
     if (splits > 65535) return TILEMIX_ERR_UNSUPPORTED;
     g->n_splits = splits;
-    g->n_parts = umma ? 2 * splits : splits;
+    g->n_parts = umma ? 2 * (g->balanced ? g->split_cap : splits) : splits;
     const size_t rows = static_cast<size_t>(p->batch) * p->heads_q * g->n_parts;
     g->o_bytes = (rows * p->head_dim * sizeof(float) + 255) / 256 * 256;
     g->mz_bytes = (rows * sizeof(float) + 255) / 256 * 256;
@@ -575,6 +607,8 @@ int tilemix_decode_int8kv(const tilemix_decode_t* p, const void* q_f16, const vo
     prm.B = p->batch; prm.Hq = p->heads_q; prm.Hk = p->heads_kv; prm.max_len = p->max_len; prm.G = p->group;
     prm.nb = p->mask_batch; prm.W = g.W; prm.n_splits = g.n_splits; prm.n_blk = g.n_blk;
     prm.tile_n = p->tile_n;
+    prm.n_parts = g.n_parts; prm.balanced = g.balanced; prm.n_rows = p->batch * p->heads_kv;
+    prm.n_ctas = g.n_ctas; prm.split_cap = g.split_cap;
     const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(static_cast<float>(p->head_dim));
     prm.scale_log2 = scale * kLog2e;
     prm.q = static_cast<const __half*>(q_f16);

@@ -11,6 +11,10 @@ namespace tilemix {
 struct DecodeParams {
     int B, Hq, Hk, max_len, G, nb, W, n_splits, n_blk;
     int tile_n;      // tokens per scale block and per routing key tile (a multiple of the kernel's chunk)
+    int n_parts;     // partial results per query head in the workspace
+    // tcgen05 form, automatic split count: n_ctas CTAs (one wave) are shared out over the n_rows = B * Hk rows by
+    // their cost, at most split_cap to a row (n_parts = 2 * split_cap); n_splits is then not used
+    int balanced, n_rows, n_ctas, split_cap;
     float scale_log2;
     const __half* q;
     const __half* k16;
@@ -21,8 +25,8 @@ struct DecodeParams {
     const uint32_t* words;
     const int32_t* cache_len;       // clamped copy in the workspace (written by the prepare kernel)
     const int32_t* cache_len_raw;   // the caller's array
-    float* o_part;   // [B, Hq, n_splits, D]
-    float* m_part;   // [B, Hq, n_splits]
+    float* o_part;   // [B, Hq, n_parts, D]
+    float* m_part;   // [B, Hq, n_parts]
     float* z_part;
     int8_t* q8_out;
     float* qs_out;

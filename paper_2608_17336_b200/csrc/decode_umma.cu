@@ -66,6 +66,7 @@ constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kTmemCols = 512;            // S^T: four buffers of 16 columns from column 0; O of stream g: 128 + 128 g
 constexpr uint32_t kColO = 128;
 constexpr float kMoveAbove = 8.f;         // m moves when a step's maximum exceeds it by more than 2^8
+constexpr int kRowsPerLane = 5, kMaxRows = 32 * kRowsPerLane;   // rows of a batch whose splits one warp can balance
 
 struct Small {
     uint64_t full[kSlots], freeb[kSlots];
@@ -79,6 +80,8 @@ struct Small {
     float dq[8];
     uint32_t tmem_base;
     int abort_flag;
+    int row_cost[kMaxRows];               // balanced splits: cost of every (sequence, KV head) row of the batch
+    int asg[4];                           // ... and this CTA's row, split and the row's number of splits
 };
 constexpr int kSmemBytes = kOffSmall + static_cast<int>(sizeof(Small)) + 1024;   // + slack to align the base to 1 KB
 static_assert(kSmemBytes <= 227 * 1024, "shared memory of one CTA");
@@ -97,8 +100,29 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
     Small& sh = *reinterpret_cast<Small*>(sm + kOffSmall);
     float2* meta = reinterpret_cast<float2*>(sm + kOffMeta);   // x = delta_K (negative: FP16 route), y = delta_V
 
-    const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Cost of the first nb groups of one 32-group mask word: a routing group costs 2 units per tile on the INT8
+    // route (K8 + V8) and 3 on the FP16 route.  `row_words`: the mask words of a (sequence, KV head) row, or null.
+    auto row_words = [&](int bb, int hh) -> const uint32_t* {
+        return prm.words != nullptr ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : bb) * prm.Hk + hh) * prm.W : nullptr;
+    };
+    auto row_groups = [&](int bb) -> int {
+        const int l = min(max(prm.cache_len_raw[bb], 0), prm.max_len);
+        return ((l + T - 1) / T + prm.G - 1) / prm.G;
+    };
+    auto word_cost = [&](const uint32_t* wr, int w, int nb) -> int {
+        const uint32_t bits = wr != nullptr ? wr[w] & (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u)) : 0u;
+        return 3 * nb - __popc(bits);
+    };
+    // Balanced splits (one wave of CTAs over a batch of at most kMaxRows rows): thread i adds up the cost of row i.
+    if (prm.balanced && tid < prm.n_rows) {
+        const int bb = tid / prm.Hk;
+        const uint32_t* wr = row_words(bb, tid - bb * prm.Hk);
+        const int ng = row_groups(bb);
+        int c = 0;
+        for (int w = 0; 32 * w < ng; ++w) c += word_cost(wr, w, min(32, ng - 32 * w));
+        sh.row_cost[tid] = c;
+    }
     // ---- set-up that needs nothing from the kernel before this one: barriers, tensor memory -----------------
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
@@ -125,59 +149,122 @@ decode_umma_kernel(const __grid_constant__ CUtensorMap tm_k8, const __grid_const
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
-    __syncthreads();                      // barriers initialised, tensor memory allocated
+    __syncthreads();                      // barriers initialised, tensor memory allocated, row costs written
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh.tmem_base);
     auto leave = [&]() {                  // early exits: tensor memory goes back first
         __syncthreads();
         if (warp == kProducerWarp) ptx::tmem_dealloc(tmem_base, kTmemCols);
     };
+    // ---- which part of which row -------------------------------------------------------------------------------
+    // Uniform form: the grid is (splits, KV heads, sequences).  Balanced form: gridDim.x CTAs, one per SM, are
+    // shared out over the rows so that the largest cost of a CTA is as small as it can be -- with one wave the
+    // CTA with the most bytes ends last, and rows differ (cache lengths, FP16-routed groups).  Row i gets
+    // s_i = clamp(ceil(c_i / tau), 1, cap) CTAs for the smallest tau whose total fits the grid; CTAs left over
+    // leave.  Every CTA finds the same tau (one warp, a binary search over at most 15 steps).
+    int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z, row_splits = prm.n_splits;
+    if (prm.balanced) {
+        if (warp == 0) {
+            int c[kRowsPerLane], cmax = 0;
+#pragma unroll
+            for (int k = 0; k < kRowsPerLane; ++k) {
+                const int i = kRowsPerLane * lane + k;
+                c[k] = i < prm.n_rows ? sh.row_cost[i] : -1;    // -1: no such row
+                cmax = max(cmax, c[k]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cmax = max(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+            auto share = [&](int cost, int tau) -> int {        // clamp(ceil(cost / tau), 1, cap), exact
+                const int num = cost + tau - 1;
+                int q = static_cast<int>(__fdividef(static_cast<float>(num), static_cast<float>(tau)));
+                if (q * tau > num) --q;
+                else if ((q + 1) * tau <= num) ++q;
+                return min(max(q, 1), prm.split_cap);
+            };
+            auto count = [&](int tau) -> int {
+                int n = 0;
+#pragma unroll
+                for (int k = 0; k < kRowsPerLane; ++k) n += c[k] >= 0 ? share(c[k], tau) : 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+                return n;
+            };
+            int lo = 1, hi = max(cmax, 1);                      // count(hi) = number of rows <= gridDim.x
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (count(mid) <= static_cast<int>(gridDim.x)) hi = mid; else lo = mid + 1;
+            }
+            int s_k[kRowsPerLane], mine = 0;
+#pragma unroll
+            for (int k = 0; k < kRowsPerLane; ++k) { s_k[k] = c[k] >= 0 ? share(c[k], hi) : 0; mine += s_k[k]; }
+            int start = mine;                                   // inclusive scan over the lanes
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, start, o);
+                if (lane >= o) start += v;
+            }
+            start -= mine;                                      // first CTA of this lane's rows
+            if (lane == 0) sh.asg[0] = -1;
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < kRowsPerLane; ++k) {
+                const int cta = static_cast<int>(blockIdx.x) - start;
+                if (cta >= 0 && cta < s_k[k]) { sh.asg[0] = kRowsPerLane * lane + k; sh.asg[1] = cta; sh.asg[2] = s_k[k]; }
+                start += s_k[k];
+            }
+        }
+        __syncthreads();
+        const int row = sh.asg[0];
+        if (row < 0) { leave(); return; }                       // a CTA left over
+        split = sh.asg[1]; row_splits = sh.asg[2];
+        b = row / prm.Hk; hk = row - b * prm.Hk;
+    }
     // This grid may run beside the prepare kernel (programmatic dependent launch): it takes the length from the
     // caller's array with the same clamp, and waits for the prepare kernel (which clears the status record) only
     // where it is about to write that record.
     const int len = min(max(prm.cache_len_raw[b], 0), prm.max_len);
     const int n_tiles = (len + T - 1) / T;
-    const uint32_t* wrow = prm.words != nullptr
-        ? prm.words + (static_cast<int64_t>(prm.nb == 1 ? 0 : b) * prm.Hk + hk) * prm.W : nullptr;
-    // The splits of a row share its BYTES, not its tiles: a routing group costs 2 units per tile on the INT8 route
-    // (K8 + V8) and 3 on the FP16 route, and with one wave of CTAs the one with the most bytes ends last.  Split
-    // k takes the groups [bound(k C / n), bound((k + 1) C / n)), C the cost of the row and bound(x) the first
-    // group at which the running cost reaches x; every thread computes the two bounds it needs (a scan over at
-    // most W mask words).
+    const uint32_t* wrow = row_words(b, hk);
+    // The splits of a row share its BYTES, not its tiles.  Split k of n takes the groups [bound(k C / n),
+    // bound((k + 1) C / n)), C the cost of the row and bound(x) the first group at which the running cost reaches
+    // x; every thread computes the two bounds it needs (a scan over at most W mask words).
     const int n_groups = (n_tiles + prm.G - 1) / prm.G;
     auto word_bits = [&](int w) -> int { return min(32, n_groups - 32 * w); };                  // groups of word w that exist
-    auto word_cost = [&](int w, int nb) -> int {                                                  // cost of its first nb groups
-        const uint32_t bits = wrow != nullptr ? wrow[w] & (nb >= 32 ? 0xffffffffu : ((1u << nb) - 1u)) : 0u;
-        return 3 * nb - __popc(bits);
-    };
     int total = 0;
-    for (int w = 0; 32 * w < n_groups; ++w) total += word_cost(w, word_bits(w));
+    for (int w = 0; 32 * w < n_groups; ++w) total += word_cost(wrow, w, word_bits(w));
     auto bound = [&](long long x) -> int {
         if (x <= 0) return 0;
         int acc = 0, w = 0;
         for (; 32 * w < n_groups; ++w) {
-            const int c = word_cost(w, word_bits(w));
+            const int c = word_cost(wrow, w, word_bits(w));
             if (acc + c >= x) break;
             acc += c;
         }
         if (32 * w >= n_groups) return n_groups;
         const int nb = word_bits(w);
         int i = 1;
-        while (i < nb && acc + word_cost(w, i) < x) ++i;    // smallest i with the cost of i groups of this word >= x - acc
+        while (i < nb && acc + word_cost(wrow, w, i) < x) ++i;    // smallest i with the cost of i groups of this word >= x - acc
         return 32 * w + i;
     };
-    const int g0 = bound(static_cast<long long>(split) * total / prm.n_splits);
-    const int g1 = split + 1 == prm.n_splits ? n_groups : bound(static_cast<long long>(split + 1) * total / prm.n_splits);
+    const int g0 = bound(static_cast<long long>(split) * total / row_splits);
+    const int g1 = split + 1 == row_splits ? n_groups : bound(static_cast<long long>(split + 1) * total / row_splits);
     const int t0 = min(n_tiles, g0 * prm.G), t1 = min(n_tiles, g1 * prm.G);
     const int n_it = t1 - t0;
     const int n_pairs = (n_it + 1) / 2;   // the softmax warps take two key tiles per step
-    const int n_parts = kStreams * prm.n_splits;   // partial results per query head in the workspace
+    const int n_parts = prm.n_parts;      // partial results per query head in the workspace (two per split, at least)
     const int64_t out_row0 = (static_cast<int64_t>(b) * prm.Hq + hk * R) * n_parts + kStreams * split;   // + r * n_parts + stream
 
     // Query row r of this KV head: FP16 copy and blockwise INT8 (block = the row), both as K-major operand rows in
     // shared memory (to_smem), and -- from the one split of the row that starts at its first group -- the quantised
     // row and its scale to the caller's buffers.
-    const bool q_writer = g0 == 0 && (g1 > 0 || split + 1 == prm.n_splits);
+    const bool q_writer = g0 == 0 && (g1 > 0 || split + 1 == row_splits);
+    // parts of the row that no split writes (balanced form: the row has fewer splits than the workspace has room
+    // for): marked empty for the merge by the row's first split
+    if (split == 0)
+        for (int idx = tid; idx < R * (n_parts - kStreams * row_splits); idx += kThreads) {
+            const int r = idx / (n_parts - kStreams * row_splits), part = kStreams * row_splits + idx % (n_parts - kStreams * row_splits);
+            prm.m_part[(static_cast<int64_t>(b) * prm.Hq + hk * R + r) * n_parts + part] = -INFINITY;
+        }
     auto prep_query_row = [&](int r, bool to_smem) {
         const int hq = hk * R + r;
         const __half* qrow = prm.q + (static_cast<int64_t>(b) * prm.Hq + hq) * D;
@@ -685,7 +772,7 @@ int launch_r(const DecodeParams& prm, const CUtensorMap& tk8, const CUtensorMap&
         if (e != cudaSuccess) return static_cast<int>(e);
         if (dev >= 0 && dev < kMaxDev) attr_set[dev][which].store(1, std::memory_order_release);
     }
-    const dim3 grid(prm.n_splits, prm.Hk, prm.B);
+    const dim3 grid = prm.balanced ? dim3(prm.n_ctas) : dim3(prm.n_splits, prm.Hk, prm.B);
     // programmatic dependent launch: this grid's set-up overlaps the tail of the prepare kernel
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;

@@ -202,6 +202,21 @@ def test_decode_host_side_validation(lib):
     # head_dim 128 with 128-key tiles (the tcgen05 form): one wave of CTAs by default (148 SMs / 64 rows = 2 splits),
     # two partial results per split
     assert splits == 2 * 2
+    # n_splits = -1: the kernel shares the wave's CTAs out by the rows' cost, up to max(16, 8 * 2) to a row
+    shared = b.tilemix_decode_workspace_size(b.decode_problem(8, 32, 8, 128, 32768, 128, 4, n_splits=-1))
+    assert shared == 512 + 8 * 32 * (2 * 16) * (128 * 4 + 8)
+    assert lib.tilemix_decode_workspace_size(ctypes.byref(b.decode_problem(8, 32, 8, 128, 32768, 128, 4, n_splits=-2))) == 0
+    # ... where it can: not with more rows than a wave has CTAs, and not in the warp-level form
+    assert (b.tilemix_decode_workspace_size(b.decode_problem(32, 32, 8, 128, 32768, 128, 4, n_splits=-1))
+            == b.tilemix_decode_workspace_size(b.decode_problem(32, 32, 8, 128, 32768, 128, 4)))
+    assert (b.tilemix_decode_workspace_size(b.decode_problem(2, 8, 2, 64, 4096, 64, 1, n_splits=-1))
+            == b.tilemix_decode_workspace_size(b.decode_problem(2, 8, 2, 64, 4096, 64, 1)))
+    # more rows than a wave has CTAs: one split per row, nothing to share out
+    many = b.tilemix_decode_workspace_size(b.decode_problem(32, 32, 8, 128, 32768, 128, 4))
+    assert many == 256 + 256 + 32 * 32 * 2 * (128 * 4 + 8)
+    # a short cache: at least four key tiles per split
+    short = b.tilemix_decode_workspace_size(b.decode_problem(1, 8, 1, 128, 1024, 128, 1))
+    assert short == 256 + 256 + 8 * (2 * 2) * 128 * 4 + 2 * 256      # (the two float arrays are rounded up to 256 bytes)
     three = b.tilemix_decode_workspace_size(b.decode_problem(8, 32, 8, 128, 32768, 128, 4, n_splits=3))
     assert three == 512 + 8 * 32 * (2 * 3) * (128 * 4 + 8)
     for bad in (b.decode_problem(0, 32, 8, 128, 1024, 128), b.decode_problem(1, 6, 4, 128, 1024, 128),

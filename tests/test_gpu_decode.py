@@ -215,6 +215,33 @@ def test_decode_gqa_group_sizes_on_the_tcgen05_form(rep):
     _check(q, k, v, route, lens, 128, 1)
 
 
+@pytest.mark.parametrize("mask_batch", [1, 5])
+def test_decode_splits_shared_out_by_the_kernel(mask_batch):
+    """n_splits = -1 on the tcgen05 form: the CTAs of one wave are shared out over the rows by their cost.  Unequal
+    cache lengths (one long sequence, short ones, an empty one, a single key), mixed masks, per batch entry or shared:
+    the long rows get many splits (up to the cap of 16), the others one each -- every output against the oracle."""
+    lens = [16384, 300, 0, 1, 4100]
+    q, k, v, route, lens = _case(5, 8, 2, 16384, 128, 128, 2, seed=90 + mask_batch, lens=lens, f8=0.6, mask_batch=mask_batch)
+    _check(q, k, v, route, lens, 128, 2, n_splits=-1)
+
+
+def test_decode_splits_shared_out_pure_routes_and_equal_rows():
+    """n_splits = -1 with rows of equal cost (nothing to gain: every row gets the same share, CTAs are left over) and
+    with the two pure masks; all INT8 without an FP16 cache."""
+    q, k, v, route, lens = _case(3, 4, 4, 2048, 128, 128, 1, seed=95, lens=[2048, 2048, 2048])
+    _check(q, k, v, np.ones_like(route), lens, 128, 1, n_splits=-1, k16_none=True)
+    _check(q, k, v, np.zeros_like(route), lens, 128, 1, n_splits=-1)
+    _check(q, k, v, route, lens, 128, 1, n_splits=-1)
+
+
+def test_decode_splits_shared_out_falls_back_where_it_cannot():
+    """n_splits = -1 means 0 in the warp-level form and with more rows than one wave has CTAs."""
+    q, k, v, route, lens = _case(2, 4, 2, 700, 64, 64, 2, seed=96, lens=[700, 33])
+    _check(q, k, v, route, lens, 64, 2, n_splits=-1)
+    q, k, v, route, lens = _case(80, 2, 2, 256, 128, 128, 1, seed=97, lens=[256 - (i % 7) * 30 for i in range(80)])
+    _check(q, k, v, route, lens, 128, 1, n_splits=-1)
+
+
 def test_decode_at_the_bench_workload_size():
     """8 sequences x 32768 cached tokens, H_q 32 / H_k 8, d 128, G = 4, 75 % INT8 groups, ragged lengths in the last
     two sequences -- the shapes and the launch configuration (library-chosen splits) that bench.py times.  Every output
