@@ -283,33 +283,42 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     uint32_t* sched_s = reinterpret_cast<uint32_t*>(smem + C::kOffWords);
     Ctx cx{reinterpret_cast<volatile int*>(&misc[1]), prm.status, prm.wait_limit_ns};
 
-    if (threadIdx.x == 0) {
-        ptx::mbar_init(bar_q(0), 1);
-        ptx::mbar_init(bar_q(1), 1);
-        for (int i = 0; i < kBundles; ++i) {
-            // on-the-fly mode: one more arrival per quantiser warp (after it made its rows of the bundle's INT8
-            // tile, if there is one to make)
-            ptx::mbar_init(bar_full(i), OTF ? 1 + kQuantWarps : 1);
-            ptx::mbar_init(bar_empty(i), hasB ? 2 : 1);   // one arrival per MMA issuer
-            ptx::mbar_init(bar_raw(i), 2);                // K16 bytes expected + "INT8 chunk claimed"
+    // Set-up, shared out so that no thread does two things in a row: lane 0 of warp 0 initialises the two "Q landed"
+    // barriers and starts the copies of the query tiles at once (they depend on nothing else and land while the rest
+    // is set up), the other lanes of warp 0 initialise one barrier each, the warps behind it build the schedule
+    // table, the first issuer warp allocates the tensor memory.
+    if (warp == 0) {
+        if (lane == 0) {
+            ptx::mbar_init(bar_q(0), 1);
+            ptx::mbar_init(bar_q(1), 1);
+            misc[1] = 0;
+        } else if (lane <= 3 * kBundles) {
+            // on-the-fly mode: one more arrival per quantiser warp on "landed" (after it made its rows of the bundle's
+            // INT8 tile, if there is one to make); "raw": K16 bytes expected + "INT8 chunk claimed"
+            const int i = (lane - 1) / 3, which = (lane - 1) % 3;
+            if (which == 0) ptx::mbar_init(bar_full(i), OTF ? 1 + kQuantWarps : 1);
+            else if (which == 1) ptx::mbar_init(bar_empty(i), hasB ? 2 : 1);   // one arrival per MMA issuer
+            else ptx::mbar_init(bar_raw(i), 2);
+        } else if (lane <= 3 * kBundles + 2) {
+            ptx::mbar_init(bar_q8(lane - 3 * kBundles - 1), kQuantWarps);
+        } else if (lane <= 3 * kBundles + 6) {
+            const int th = lane - 3 * kBundles - 3;
+            ptx::mbar_init(bar_s(th >> 1, th & 1), 1);
+        } else if (lane <= 3 * kBundles + 10) {
+            const int th = lane - 3 * kBundles - 7;
+            ptx::mbar_init(bar_p(th >> 1, th & 1), kSoftmaxWarps / 2 * 32);
+        } else if (lane <= 3 * kBundles + 12) {
+            ptx::mbar_init(bar_pv(lane - 3 * kBundles - 11), 1);
+        } else if (lane <= 3 * kBundles + 14) {
+            ptx::mbar_init(bar_o(lane - 3 * kBundles - 13), 1);
+        } else if (lane == 3 * kBundles + 15) {
+            ptx::mbar_init(bar_drain, hasB ? 2 : 1);
         }
-        ptx::mbar_init(bar_q8(0), kQuantWarps);
-        ptx::mbar_init(bar_q8(1), kQuantWarps);
-        for (int t = 0; t < 2; ++t) {
-            for (int h = 0; h < 2; ++h) {
-                ptx::mbar_init(bar_s(t, h), 1);
-                ptx::mbar_init(bar_p(t, h), kSoftmaxWarps / 2 * 32);
-            }
-            ptx::mbar_init(bar_pv(t), 1);
-            ptx::mbar_init(bar_o(t), 1);
-        }
-        ptx::mbar_init(bar_drain, hasB ? 2 : 1);
-        misc[1] = 0;
+        static_assert(3 * kBundles + 15 < 32, "one barrier per lane of warp 0");
         ptx::fence_mbar_init();
-        s_skip = skip_word;
-        // The query tiles do not depend on the schedule table: their copies start here, ahead of the set-up
-        // barrier, and land while the table is being built.
-        if (skip_word == 0) {
+        if (lane == 0) {
+            // The copies start whatever the status word says (its load is still on its way): a CTA that then finds
+            // it has nothing to do waits for them before it leaves.
             for (int t = 0; t < (hasB ? 2 : 1); ++t) {
                 const int m = t ? mB : mA;
                 const uint32_t bytes = C::kQ16Tile + ((prm.has_int8 && !OTF) ? C::kQ8Tile : 0);
@@ -320,24 +329,37 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (prm.has_int8 && !OTF)
                     ptx::tma_load_4d(sbase + C::kOffQ8 + t * C::kQ8Tile, &tm_q8, bar_q(t), 0, tok0 + m * T, hq, b);
             }
+            s_skip = skip_word;
         }
     }
     // Schedule table, one 4-bit entry per key tile j (Sec. 4.2 lookup done once per CTA):
     //   bit0 / bit1: tile A / tile B takes the INT8 route at key tile j  (R = (b >> floor(j/G)) & 1)
     //   bit2 / bit3: the FP16 / the INT8 copy of K_j has to be staged
-    for (int i = threadIdx.x; i * 8 < nkv; i += blockDim.x) {
+    // A thread makes eight consecutive entries.  Their groups lie in at most two mask words per row: the four words
+    // are loaded up front, so that the thread waits for one round trip, not for one per entry.
+    for (int i = static_cast<int>(threadIdx.x) - 32; i >= 0 && i * 8 < nkv; i += static_cast<int>(blockDim.x) - 32) {
+        const int j0 = i * 8, j_last = min(j0 + 7, nkv - 1);
+        int g = 0, in_g = 0, w_lo = 0;
+        uint32_t wa[2] = {0u, 0u}, wb[2] = {0u, 0u};
+        if (prm.words != nullptr) {
+            g = j0 / prm.G;
+            in_g = j0 - g * prm.G;
+            w_lo = g >> 5;
+            const int w_hi = (j_last / prm.G) >> 5;
+            const int nbi = (prm.nb == 1) ? 0 : b;
+            const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.mask_T_m + row0 + mA) * prm.W;
+            wa[0] = rowA[w_lo];
+            wa[1] = rowA[w_hi];
+            if (hasB) { wb[0] = rowA[prm.W + w_lo]; wb[1] = rowA[prm.W + w_hi]; }
+        }
         uint32_t packed = 0u;
         for (int jj = 0; jj < 8; ++jj) {
-            const int j = i * 8 + jj;
-            if (j >= nkv) break;
-            uint32_t e = 0u;
-            if (prm.words != nullptr) {
-                const int g = j / prm.G;
-                const int nbi = (prm.nb == 1) ? 0 : b;
-                const uint32_t* rowA = prm.words + ((static_cast<int64_t>(nbi) * prm.Hk + hk) * prm.mask_T_m + row0 + mA) * prm.W;
-                e |= (rowA[g >> 5] >> (g & 31)) & 1u;
-                if (hasB) e |= ((rowA[prm.W + (g >> 5)] >> (g & 31)) & 1u) << 1;
-            }
+            const int j = j0 + jj;
+            if (j > j_last) break;
+            const bool hi = (g >> 5) != w_lo;              // (no mask words: all bits 0)
+            uint32_t e = ((hi ? wa[1] : wa[0]) >> (g & 31)) & 1u;
+            if (hasB) e |= (((hi ? wb[1] : wb[0]) >> (g & 31)) & 1u) << 1;
+            if (++in_g == prm.G) { in_g = 0; ++g; }
             const bool useA = j <= kA;
             if ((useA && !(e & 1u)) || (hasB && !(e & 2u))) e |= 4u;
             if ((useA && (e & 1u)) || (hasB && (e & 2u))) e |= 8u;
@@ -354,7 +376,11 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = misc[0];
-    if (s_skip != 0) {   // nothing is in flight (no copy was started): give the tensor memory back and leave
+    if (s_skip != 0) {   // only the query tiles are in flight: let them land, give the tensor memory back and leave
+        if (threadIdx.x == 0)
+            for (int t = 0; t < (hasB ? 2 : 1); ++t)
+                for (int it = 0; it < (1 << 20); ++it)
+                    if (ptx::mbar_try_wait(bar_q(t), 0)) break;
         if (warp == kMmaWarp) ptx::tmem_dealloc(tmem_base, C::kTmemCols);
         return;
     }
