@@ -307,10 +307,28 @@ def decode_leg(tm, w: synth.Workload, dev, peaks) -> dict:
     # algorithmic bytes: per cached token d (V8) + d (K8, INT8 route) or 2d (FP16 K, FP16 route)
     nbytes = float(B) * Hk * L * d * (1.0 + f8 + 2.0 * (1.0 - f8))
     gbs = nbytes / (ms * 1e-3) / 1e9
-    return {"batch": B, "heads_q": Hq, "heads_kv": Hk, "cache_len": L, "int8_groups": f8, "ms_per_step": ms,
-            "tokens_per_s": B / (ms * 1e-3), "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
-            "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "bytes_per_step": nbytes,
-            "l2": "cache (0.8 GB) exceeds L2"}
+    res = {"batch": B, "heads_q": Hq, "heads_kv": Hk, "cache_len": L, "int8_groups": f8, "ms_per_step": ms,
+           "tokens_per_s": B / (ms * 1e-3), "bound": "hbm", "achieved": gbs, "peak": float(peaks["hbm_gbs"]),
+           "unit": "GB/s", "frac": gbs / float(peaks["hbm_gbs"]), "bytes_per_step": nbytes,
+           "l2": "cache (0.8 GB) exceeds L2"}
+    # the same cache with unequal lengths: the library's uniform split count against splits shared out over the
+    # rows by the kernel (n_splits = -1)
+    ragged = [L, L // 8, L // 16, L // 2, L // 32, L // 4, L // 64, (3 * L) // 4]
+    lens_r = torch.tensor(ragged, dtype=torch.int32, device=dev)
+    res["unequal_lengths"] = {"cache_len": ragged}
+    for key, ns in (("uniform_splits_ms", 0), ("kernel_chosen_splits_ms", -1)):
+        pr = tm.decode_problem(B, Hq, Hk, d, L, w.tile, w.group, n_splits=ns)
+        work_r = torch.empty(tm.tilemix_decode_workspace_size(pr), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            tm.tilemix_decode_int8kv(pr, q, k, k8, ks, v8, vs, words_d, lens_r, out=out, workspace=work_r)
+        torch.cuda.synchronize()
+        t0.record(stream)
+        for _ in range(n):
+            tm.tilemix_decode_int8kv(pr, q, k, k8, ks, v8, vs, words_d, lens_r, out=out, workspace=work_r)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        res["unequal_lengths"][key] = t0.elapsed_time(t1) / n
+    return res
 
 
 def main():
