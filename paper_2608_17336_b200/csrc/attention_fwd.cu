@@ -189,7 +189,10 @@ struct Ring {
 // OTF: on-the-fly operand generation (App. D, "fused on-the-fly" mode): there are no INT8 copies of Q and K
 // and no scales in global memory; a quantiser warp makes them in shared memory from the FP16 tiles, for
 // the key tiles some query tile of the CTA routes to INT8 only.
-template <int D, int T, bool VL, bool OTF, bool VS = false>
+// DBG: the instance that can write the raw accumulators of requested tiles (every step then takes the generic form).
+// A kernel of its own, because every instruction in the softmax warps' loop that is not executed still costs: the loop
+// of the other instances is ~1 % faster without that code in it.
+template <int D, int T, bool VL, bool OTF, bool VS = false, bool DBG = false>
 __global__ void __launch_bounds__(OTF ? kThreadsOtf : kThreads, 1)
 attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                  const __grid_constant__ CUtensorMap tm_k16, const __grid_constant__ CUtensorMap tm_v16,
@@ -810,7 +813,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
 
                 // P = 2^(a*raw - m) is rounded to FP16, one pair per register.
                 const bool diag = (j == k_t);
-                bool redo = diag || u == 0 || prm.dbg_n > 0;
+                bool redo = diag || u == 0 || DBG;
                 bool stored = false;      // P of the one-pass form has been sent to tensor memory
                 float alpha[2] = {1.f, 1.f}, sum[2] = {0.f, 0.f};
                 bool grow = false;
@@ -838,7 +841,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                 if (redo) {
                     // Generic two-pass form: the very first step, the diagonal tile, steps that move the maximum, and
                     // every step in debug mode.
-                    if (prm.dbg_n > 0) {   // debug mode: raw accumulators of the requested tiles
+                    if constexpr (DBG) {   // debug mode: raw accumulators of the requested tiles
                         int idx = -1;
                         if (lane == 0) {
                             for (int e = 0; e < prm.dbg_n; ++e) {
@@ -917,7 +920,7 @@ attention_kernel(const Params prm, const __grid_constant__ CUtensorMap tm_q16,
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 1                     // (rare: kept small, see DBG above)
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[16];
                         ptx::tmem_ld16x256_x4(t_o + c * 32, o);
@@ -1078,11 +1081,16 @@ int launch_impl(const Geometry& g, const void* q, const void* k, const void* v, 
     }
     cudaError_t e = cudaMemsetAsync(workspace, 0, kWorkspaceClearBytes, stream);
     if (e != cudaSuccess) return static_cast<int>(e);
-    auto kernel = vl ? attention_kernel<D, T, true, false> : attention_kernel<D, T, false, false>;
+    const bool dbg_on = prm.dbg_n > 0;
+    auto kernel = vl ? (dbg_on ? attention_kernel<D, T, true, false, false, true> : attention_kernel<D, T, true, false>)
+                     : (dbg_on ? attention_kernel<D, T, false, false, false, true> : attention_kernel<D, T, false, false>);
     if constexpr (D == 128 && T == 128) {
-        if (otf) kernel = attention_kernel<D, T, false, true>;
+        if (otf) kernel = dbg_on ? attention_kernel<D, T, false, true, false, true> : attention_kernel<D, T, false, true>;
     }
-    if (v_scale != nullptr) kernel = attention_kernel<D, T, false, false, true>;
+    if (v_scale != nullptr) {
+        if (dbg_on) return TILEMIX_ERR_UNSUPPORTED;     // (the chunk against an INT8 value cache has no debug instance)
+        kernel = attention_kernel<D, T, false, false, true>;
+    }
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemAlloc);
     if (e != cudaSuccess) return static_cast<int>(e);
     const int64_t ctas = vl ? static_cast<int64_t>(g.Hq) * total_pairs
