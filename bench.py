@@ -31,8 +31,8 @@ METRIC = "effective causal-attention TFLOP/s at 1 B200 vs INT8 fraction; % of mi
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_FP16 = 2.0     # nominal dense INT8 : FP16 tensor throughput ratio (4.5 : 2.25 PFLOP/s)
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from an ncu capture of the 8-head case of
-# the workload (492.3 MB; the traffic scales with the head count).
-NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 492.3e6 / 8}
+# the workload (484.1 MB; the traffic scales with the head count).
+NCU_DRAM_BYTES_PER_HEAD = {"cfg3_long32k": 484.1e6 / 8}
 
 
 def effective_flops(w: synth.Workload) -> float:
