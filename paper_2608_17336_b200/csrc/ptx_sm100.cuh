@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the attention kernel uses: mbarrier,
-// TMA tiled loads (no multicast), tcgen05 (TMEM allocation, MMA, commit, load/store, fences).
+// TMA tiled loads (each CTA fetches its own tiles), tcgen05 (TMEM allocation, MMA, commit, load/store, fences).
 #pragma once
 
 #include <cuda.h>
@@ -68,7 +68,7 @@ __device__ __forceinline__ void tc_fence_after_sync() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-// ---------------------------------------------------------------- TMA (tiled, 4-D, no multicast)
+// ---------------------------------------------------------------- TMA (tiled, 4-D, one destination CTA)
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
 }
@@ -82,7 +82,7 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm,
         : "memory");
 }
 
-// Untiled bulk copy global -> shared memory (no multicast): both addresses 16-byte aligned, `bytes` a
+// Untiled bulk copy global -> shared memory (one destination CTA): both addresses 16-byte aligned, `bytes` a
 // multiple of 16; completion is counted in bytes on the mbarrier.
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile(
